@@ -1,0 +1,379 @@
+#!/usr/bin/env python
+"""Benchmark of the verify pass: ``python bench.py --gpus N --steps K --warmup W``.
+
+A step is one whole verify pass (nested-prefix attention -> greedy acceptance ->
+commit) over one batch of seeded synthetic input.  The workload is the
+"32B-class single attention layer" configuration unless ``--config`` says
+otherwise.  Every rank owns an independent batch (requests do not interact, so
+the path shards by request with no collective: weak scaling).
+
+Cold-HBM protocol: the KV pools and the logits exist in ``--copies`` independent
+copies whose total footprint is several times the L2; step i uses copy i mod
+copies, so every step streams its inputs from HBM.
+
+``--impl reference`` times the CPU fp64 oracle (there is no other implementation
+of this path to run) on the host cores, on the same workload and metric.
+"""
+from __future__ import annotations
+
+import argparse
+import ctypes
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "verified_tokens_per_s_per_verify_pass"
+UNIT = "tokens/s"
+FALLBACK_HBM_GBS = 6650.0
+FALLBACK_BF16_TFLOPS = 1590.0
+
+
+def _peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            d = json.load(open(p))
+            return float(d["hbm_gbs"]), float(d["bf16_tflops"]), "measured"
+        except Exception:
+            pass
+    return FALLBACK_HBM_GBS, FALLBACK_BF16_TFLOPS, "fallback"
+
+
+def attention_work(batch):
+    """Algorithmic bytes and flops of the attention step: every KV row of every span and tail once
+    (K and V), Q read and O written once; 4*D flops per (query row, head, visible key)."""
+    m = batch.model
+    kv_bytes = batch.kv_tokens() * m.n_kv_heads * m.head_dim * 2 * 2
+    qo_bytes = 2 * batch.n_q_rows * m.n_q_heads * m.head_dim * 2
+    vis = 0
+    for b in range(batch.n_branch):
+        r = int(batch.br_req[b])
+        s0 = int(batch.req_span_off[r])
+        chain = int(batch.span_len[s0 : s0 + 1 + int(batch.br_depth[b])].sum())
+        q_len = int(batch.cu_q[b + 1] - batch.cu_q[b])
+        own = int(batch.br_own_len[b])
+        vis += sum(chain + own - q_len + i + 1 for i in range(q_len))
+    flops = 4 * m.n_q_heads * m.head_dim * vis
+    return kv_bytes + qo_bytes, flops
+
+
+def accept_bytes(batch):
+    return batch.n_logit_rows * batch.model.vocab * 2
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons every 200 ms while the timed region runs."""
+
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.gpu = gpu_index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "200", "-i", str(self.gpu)],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.25)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def oracle_pass_seconds(w, min_seconds, max_passes=1000):
+    """Times whole oracle passes on workload w until min_seconds of CPU work are done."""
+    from oracle import lr_oracle as O
+
+    b, t = w.batch, w.tensors
+    n, t0 = 0, time.perf_counter()
+    while True:
+        O.verify_pass(b, t.q, t.k_pool, t.v_pool, t.logits, t.draft_ids, t.verdict)
+        n += 1
+        el = time.perf_counter() - t0
+        if el >= min_seconds or n >= max_passes:
+            return el / n, n
+
+
+def host_threads():
+    try:
+        from threadpoolctl import threadpool_info
+
+        n = max([p.get("num_threads", 1) for p in threadpool_info()] or [1])
+        return int(n)
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def run_reference(args):
+    """The reference arm: the CPU oracle, as it stands, on the host cores."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    from lr_workloads import make_config
+
+    w = make_config(args.config)
+    tokens = w.batch.n_verified_tokens
+    for _ in range(args.warmup):
+        oracle_pass_seconds(w, 0.0, 1)
+    times = []
+    budget_end = time.perf_counter() + 150.0
+    for _ in range(args.steps):
+        s, _ = oracle_pass_seconds(w, 0.0, 1)
+        times.append(s)
+        if time.perf_counter() > budget_end:
+            break
+    sec = sum(times) / len(times)
+    cores = host_threads()
+    val = tokens / sec
+    sample = f"whole pass of config {args.config} ({w.name}), one batch per step, {len(times)} steps"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": len(times),
+        "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic", "config": {"workload": f"config{args.config}_{w.name}", "seed": w.seed},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=400)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=2)
+    ap.add_argument("--copies", type=int, default=0, help="independent copies of pools/logits (0 = enough for 6x L2)")
+    ap.add_argument("--cpu-seconds", type=float, default=12.0)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--path", type=int, default=0, help="attention path: 0 auto, 1 CUDA cores, 2 tensor cores")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+
+    import torch
+    import torch.distributed as dist
+
+    from lr_workloads import make_config
+    from paper_2506_19830_b200 import binding as B
+    from paper_2506_19830_b200 import runner as R
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the verify pass has no CPU path")
+    torch.cuda.set_device(local)
+    dev = f"cuda:{local}"
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+
+    w = make_config(args.config, seed=20250619 + args.config + 1000 * rank)
+    b, t = w.batch, w.tensors
+    ctx = B.Context(b.model, local)
+    plan = B.Plan(ctx, b)
+    plan.lr_plan_set_attention_path(args.path)
+    x0 = R.DeviceInputs(b, t, dev)
+    y = R.PassOutputs(b, dev)
+    per_copy = 2 * x0.k_pool.numel() * 2 + x0.logits.numel() * 2
+    copies = args.copies if args.copies > 0 else max(4, int(np.ceil(6 * 126e6 / per_copy)))
+    copies = min(copies, max(1, int(40e9 // per_copy)))
+    kc = [x0.k_pool] + [x0.k_pool.clone() for _ in range(copies - 1)]
+    vc = [x0.v_pool] + [x0.v_pool.clone() for _ in range(copies - 1)]
+    lc = [x0.logits] + [x0.logits.clone() for _ in range(copies - 1)]
+    stream = torch.cuda.current_stream()
+
+    def step(i):
+        c = i % copies
+        plan.lr_verify_attention(x0.q, kc[c], vc[c], y.out, None, 0.0, stream)
+        ctx.lr_accept_greedy(lc[c], x0.draft_ids, x0.cu_draft, y.n_accept, y.bonus_id, y.scratch, None, stream)
+        plan.lr_commit(x0.verdict, y.n_accept, y.n_steps_accepted, y.survivor, y.committed_len, y.keep_off, y.keep_pages,
+                       y.keep_valid, y.free_off, y.free_pages, stream)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    W = max(args.warmup, 3)
+    K = args.steps
+    for i in range(W):
+        step(i)
+    assert plan.lr_poll_status() == 0
+
+    # ---- region A: K whole steps, device time -------------------------------------
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    launches0 = ctx.launch_count
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record(stream)
+    for i in range(K):
+        step(W + i)
+    e1.record(stream)
+    barrier()
+    launches = ctx.launch_count - launches0
+    ms_total = e0.elapsed_time(e1)
+
+    # ---- region B: the same K steps with an event pair around every launch --------
+    names = ("attention", "accept", "commit")
+    ev = {n: [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)] for n in names}
+    barrier()
+    for i in range(K):
+        c = (W + i) % copies
+        a, z = ev["attention"][i]
+        a.record(stream)
+        plan.lr_verify_attention(x0.q, kc[c], vc[c], y.out, None, 0.0, stream)
+        z.record(stream)
+        a, z = ev["accept"][i]
+        a.record(stream)
+        ctx.lr_accept_greedy(lc[c], x0.draft_ids, x0.cu_draft, y.n_accept, y.bonus_id, y.scratch, None, stream)
+        z.record(stream)
+        a, z = ev["commit"][i]
+        a.record(stream)
+        plan.lr_commit(x0.verdict, y.n_accept, y.n_steps_accepted, y.survivor, y.committed_len, y.keep_off, y.keep_pages,
+                       y.keep_valid, y.free_off, y.free_pages, stream)
+        z.record(stream)
+    barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    kernel_us = {n: 1e3 * sum(a.elapsed_time(z) for a, z in ev[n]) / K for n in names}
+    assert plan.lr_poll_status() == 0
+
+    # ---- end to end: host buffers in, host results out -----------------------------
+    e2e = None
+    if not args.no_e2e:
+        m = b.model
+        pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()  # noqa: E731
+        host = {
+            "q_h": pin(t.q.view(np.int16)), "logits_h": pin(t.logits.view(np.int16)), "draft_ids_h": pin(t.draft_ids),
+            "verdict_h": pin(t.verdict if len(t.verdict) else np.zeros(1, np.uint8)),
+            "out_h": torch.empty((b.n_q_rows, m.n_q_heads, m.head_dim), dtype=torch.int16).pin_memory(),
+        }
+        for name, n in (("n_accept_h", b.n_branch), ("bonus_id_h", b.n_branch), ("n_steps_accepted_h", b.n_req),
+                        ("survivor_h", b.n_req), ("committed_len_h", b.n_req), ("keep_off_h", b.n_req + 1),
+                        ("free_off_h", b.n_req + 1), ("keep_pages_h", b.n_page_slots), ("keep_valid_h", b.n_page_slots),
+                        ("free_pages_h", b.n_page_slots)):
+            host[name] = torch.empty(n, dtype=torch.int32).pin_memory()
+        io = B.lr_pass_host_io(**{k: v.data_ptr() for k, v in host.items()})
+        staging = plan.pass_staging()
+        h2d = sum(host[k].numel() * host[k].element_size() for k in ("q_h", "logits_h", "draft_ids_h", "verdict_h"))
+        d2h = sum(v.numel() * v.element_size() for k, v in host.items() if k not in ("q_h", "logits_h", "draft_ids_h", "verdict_h"))
+        Ke = max(3, min(K, 50))
+        for i in range(3):
+            plan.lr_verify_pass_host(io, kc[i % copies], vc[i % copies], staging, 0.0, stream)
+        barrier()
+        t0 = time.perf_counter()
+        for i in range(Ke):
+            plan.lr_verify_pass_host(io, kc[(W + i) % copies], vc[(W + i) % copies], staging, 0.0, stream)
+        torch.cuda.synchronize()
+        e2e_s = (time.perf_counter() - t0) / Ke
+        e2e_t = torch.tensor([e2e_s], device=dev, dtype=torch.float64)
+        if world > 1:
+            dist.all_reduce(e2e_t, op=dist.ReduceOp.MAX)
+        e2e = {"value": world * b.n_verified_tokens / float(e2e_t.item()), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
+               "d2h_bytes_per_step": int(d2h), "ms_per_step": float(e2e_t.item()) * 1e3, "steps": Ke,
+               "note": "lr_verify_pass_host: pinned host Q/logits/drafts/verdicts in, all results out, stream sync per step; "
+                       "KV pools are device-resident cache state"}
+
+    # ---- aggregate over ranks --------------------------------------------------------
+    tmax = torch.tensor([ms_total], device=dev, dtype=torch.float64)
+    tok = torch.tensor([float(b.n_verified_tokens)], device=dev, dtype=torch.float64)
+    if world > 1:
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+        dist.all_reduce(tok, op=dist.ReduceOp.SUM)
+    ms_step = float(tmax.item()) / K
+    value = float(tok.item()) / (ms_step * 1e-3)
+
+    if rank == 0:
+        hbm_peak, tc_peak, peak_kind = _peaks()
+        a_bytes, a_flops = attention_work(b)
+        t_att = kernel_us["attention"] * 1e-6
+        hbm_time, tc_time = a_bytes / (hbm_peak * 1e9), a_flops / (tc_peak * 1e12)
+        if hbm_time >= tc_time:
+            roof = {"bound": "hbm", "achieved": a_bytes / t_att / 1e9, "peak": hbm_peak, "unit": "GB/s"}
+        else:
+            roof = {"bound": "tensor", "achieved": a_flops / t_att / 1e12, "peak": tc_peak, "unit": "TFLOP/s"}
+        roof["frac"] = roof["achieved"] / roof["peak"]
+        roof.update({"traffic": None, "kernel": "lr_verify_attention", "kernel_us": kernel_us["attention"],
+                     "algorithmic_bytes": a_bytes, "algorithmic_flops": a_flops, "peak_source": f"of {peak_kind}",
+                     "roofline_us": max(hbm_time, tc_time) * 1e6})
+        acc_b = accept_bytes(b)
+        kernels = {
+            "lr_verify_attention": {"us": kernel_us["attention"], "GB/s": a_bytes / t_att / 1e9,
+                                    "TFLOP/s": a_flops / t_att / 1e12},
+            "lr_accept_greedy": {"us": kernel_us["accept"], "GB/s": acc_b / (kernel_us["accept"] * 1e-6) / 1e9,
+                                 "frac_of_hbm_peak": acc_b / (kernel_us["accept"] * 1e-6) / 1e9 / hbm_peak,
+                                 "algorithmic_bytes": acc_b},
+            "lr_commit": {"us": kernel_us["commit"]},
+        }
+        cpu = None
+        if not args.no_cpu_baseline:
+            sec, n = oracle_pass_seconds(w, args.cpu_seconds)
+            cpu = {"value": b.n_verified_tokens / sec, "unit": UNIT, "cores": host_threads(), "kind": "oracle",
+                   "sample": f"{n} whole passes of the same workload (config {args.config}), {sec * 1e3:.1f} ms each",
+                   "ms_per_pass": sec * 1e3}
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W, "ms_per_step": ms_step,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": f"config{args.config}_{w.name}", "seed": w.seed, "requests_per_gpu": b.n_req,
+                       "branches_per_gpu": b.n_branch, "kv_tokens_per_gpu": b.kv_tokens(), "verified_tokens_per_gpu": b.n_verified_tokens,
+                       "l2_policy": f"rotating {copies} copies of KV pools and logits ({copies * per_copy / 1e6:.0f} MB > L2)",
+                       "attention_path": args.path},
+            "roofline": roof, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
+            "kernels": kernels,
+        }
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -1,0 +1,244 @@
+/*
+ * lr_verify.h -- C ABI of the step-parallel verification pass of Lookahead
+ * Reasoning on one B200 (sm_100a).
+ *
+ * One verify pass (Algorithm 1, the "in parallel do" block, with token-level
+ * speculative decoding running inside every branch) is three device steps:
+ *
+ *   lr_verify_attention  nested-prefix paged GQA attention of every branch's
+ *                        query tokens over  prefix (+) S_1..S_depth (+) own tail
+ *   lr_accept_greedy     greedy token-level acceptance over vocab-wide logits
+ *   lr_commit            step-level output construction on the paged KV cache
+ *
+ * Conventions
+ *   - Plain C.  No exceptions, no aborts, no device traps.  Every function
+ *     returns LR_OK (0) or a negative lr_status; lr_strerror() names it and
+ *     lr_last_error() gives the detail message of the calling thread's last
+ *     failing call.
+ *   - Pointers ending in _h are HOST pointers, pointers ending in _d are DEVICE
+ *     pointers on the context's device.  All buffers are owned by the caller;
+ *     the library never frees or reallocates them.  The only device memory the
+ *     library itself ever uses is inside the caller-provided workspace /
+ *     scratch buffers; host-side it owns the opaque lr_ctx / lr_plan objects.
+ *   - "stream" is a cudaStream_t passed as void*.  All device work is enqueued
+ *     on it and no call synchronises unless its comment says so.
+ *   - bf16 tensors are passed as raw pointers to 16-bit words.
+ *   - There is no CPU fallback: without a usable sm_100 device every call fails.
+ *   - Same inputs and same plan give bit-identical outputs.
+ *
+ * Data layout
+ *   Q, O      [n_q_rows][n_q_heads][head_dim] bf16, rows packed by branch
+ *             (branch b owns rows cu_q[b] .. cu_q[b+1]-1, in token order).
+ *   K/V pool  [n_pool_pages][n_kv_heads][16][head_dim] bf16; a page holds 16
+ *             tokens.  Every span (prefix, segment, tail) starts at token slot 0
+ *             of its first page and owns whole pages; the unused slots of its
+ *             last page may hold anything (NaN included) and never affect a
+ *             result.  A physical page belongs to at most one span.
+ *   logits    [n_rows][row_stride] bf16, first `vocab` entries of a row used;
+ *             branch b with L_b drafts owns the L_b+1 rows starting at
+ *             cu_draft[b] + b: row i scores draft i, row L_b gives the bonus.
+ */
+#ifndef LR_VERIFY_H_
+#define LR_VERIFY_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum lr_status {
+  LR_OK = 0,
+  LR_EINVAL = -1,       /* bad argument: null pointer, inconsistent lengths, page id out of range ... */
+  LR_EUNSUPPORTED = -2, /* shape or device outside what the kernels implement */
+  LR_ECUDA = -3,        /* a CUDA runtime / driver call failed (text in lr_last_error) */
+  LR_ETIMEOUT = -4,     /* a bounded device-side wait expired (reported by lr_poll_status) */
+  LR_EBOUNDS = -5,      /* a device-side bounds check tripped (reported by lr_poll_status) */
+  LR_ENOMEM = -6        /* caller-provided workspace too small / host allocation failed */
+} lr_status;
+
+typedef struct lr_ctx lr_ctx;   /* per (device, model geometry) */
+typedef struct lr_plan lr_plan; /* per batch structure; reusable across passes and KV pools */
+
+/* Model geometry.  Supported: head_dim 64 or 128, page_size 16,
+ * n_q_heads a multiple of n_kv_heads with group size <= 16, vocab >= 1. */
+typedef struct lr_model {
+  int32_t n_q_heads, n_kv_heads, head_dim, page_size, vocab;
+} lr_model;
+
+/*
+ * Integer description of one pass; every array is a HOST array of int32 that
+ * only needs to live until lr_plan_create returns.
+ *
+ * Request r owns chain spans req_span_off[r] .. req_span_off[r+1]-1: the first
+ * is the shared prefix x_{1:t} (length >= 0), the c-th after it is draft step
+ * segment c (length >= 1), c = 1..gamma_r.  Span s holds span_len[s] tokens in
+ * page slots span_slot[s] .. span_slot[s]+ceil(len/16)-1 of page_ids[].
+ *
+ * Branch b (branches of one request are contiguous, br_req non-decreasing)
+ * sees the prefix and the first br_depth[b] segments of its request (that is
+ * x'_j of Algorithm 1 with j = depth) plus, causally, its private tail of
+ * br_own_len[b] tokens (slots from br_own_slot[b]); the LAST q_len_b =
+ * cu_q[b+1]-cu_q[b] tail tokens are the queries.  br_n_draft[b] (<= own_len)
+ * is L_b, the number of token-level drafts being verified for the branch.
+ */
+typedef struct lr_batch {
+  int32_t n_req, n_branch, n_span, n_page_slots;
+  const int32_t *req_span_off; /* [n_req+1]   */
+  const int32_t *span_len;     /* [n_span]    */
+  const int32_t *span_slot;    /* [n_span]    */
+  const int32_t *br_req;       /* [n_branch]  */
+  const int32_t *br_depth;     /* [n_branch]  0..gamma_r */
+  const int32_t *br_own_len;   /* [n_branch]  >= q_len   */
+  const int32_t *br_own_slot;  /* [n_branch]  */
+  const int32_t *br_n_draft;   /* [n_branch]  0..own_len */
+  const int32_t *cu_q;         /* [n_branch+1] query-row offsets, q_len >= 1 */
+  const int32_t *page_ids;     /* [n_page_slots] physical page numbers, distinct */
+  int64_t n_pool_pages;        /* pages in each of the K and V pools */
+} lr_batch;
+
+/* Host-only check of a batch description against the rules above (no device
+ * needed): LR_OK, or LR_EINVAL with the first violated rule in lr_last_error(). */
+int lr_validate_batch(const lr_model *model, const lr_batch *batch_h);
+
+/* ---- context ------------------------------------------------------------ */
+
+/* Creates a context on CUDA device `device` (must be compute capability 10.x).
+ * Allocates only host memory.  LR_EUNSUPPORTED for geometry outside the list
+ * above or a non-sm_100 device. */
+int lr_create(lr_ctx **out, const lr_model *model, int device);
+int lr_destroy(lr_ctx *ctx);
+
+/* ---- plan --------------------------------------------------------------- */
+
+/* Bytes of device workspace lr_plan_create needs for this batch (metadata
+ * tables, the work list of the attention kernel, split-KV partial results and
+ * a status word).  Validates the batch (LR_EINVAL with detail on failure). */
+int lr_plan_bytes(const lr_ctx *ctx, const lr_batch *batch_h, size_t *bytes_out);
+
+/* Validates the batch, builds the device-side tables and the attention work
+ * partition on the host and enqueues their upload into workspace_d (256-byte
+ * aligned, >= lr_plan_bytes) on `stream`.  The host staging copy lives in the
+ * plan, so the call does not synchronise.  The plan may be used by any number
+ * of later passes over any KV pools with >= batch_h->n_pool_pages pages, on
+ * the same stream (or after the upload has completed).  Two passes that use
+ * the same plan must not overlap on the device (they share the workspace). */
+int lr_plan_create(lr_ctx *ctx, const lr_batch *batch_h, void *workspace_d, size_t workspace_bytes,
+                   void *stream, lr_plan **out);
+int lr_plan_destroy(lr_plan *plan);
+
+/* ---- the three steps ---------------------------------------------------- */
+
+/*
+ * Nested-prefix verify attention (Algorithm 1, parallel target step generation;
+ * Background, "verifies these tokens in a single parallel forward pass").
+ * For every branch b, query i, head h:
+ *     O = softmax(scale * q K^T) V   over the keys of the prefix, of segments
+ *     1..depth_b and of tail tokens 0 .. own_len_b - q_len_b + i   (inclusive),
+ * with KV head h / (n_q_heads / n_kv_heads).  softmax_scale <= 0 selects
+ * 1/sqrt(head_dim).  out_d: [n_q_rows][n_q_heads][head_dim] bf16.  lse_d
+ * (nullable): [n_q_rows][n_q_heads] fp32, natural log of the sum of exp of the
+ * scaled scores.  Accumulation and softmax are fp32.
+ * Errors: LR_EINVAL (null / misaligned pointers: q, out, pools need 16-byte
+ * alignment), LR_ECUDA (launch failure).  Device-side problems (a page id
+ * beyond the pool, an expired wait) set the plan's status word; see
+ * lr_poll_status.
+ */
+int lr_verify_attention(lr_plan *plan, const void *q_d, const void *k_pool_d, const void *v_pool_d,
+                        void *out_d, float *lse_d, float softmax_scale, void *stream);
+
+/* Selects the attention implementation for later lr_verify_attention calls on
+ * this plan: 0 = automatic (tensor-core path when the shape allows it), 1 =
+ * force the CUDA-core path (every shape), 2 = force the tensor-core path
+ * (LR_EUNSUPPORTED later if the shape does not allow it).  For testing. */
+int lr_plan_set_attention_path(lr_plan *plan, int path);
+
+/* Bytes of scratch lr_accept_greedy needs for n_rows logits rows.  The scratch
+ * must be zero-filled before its first use; every call leaves it zero-filled. */
+int lr_accept_scratch_bytes(int32_t n_rows, size_t *bytes_out);
+
+/*
+ * Greedy token-level acceptance (Background, "Speculative Decoding": drafts are
+ * processed in order, the process halts at the first rejected one and a final
+ * token comes from the target's distribution at that position).
+ *     t_i    = argmax_v logits[row0_b + i][v]      (lowest index on ties, +0 == -0,
+ *                                                   NaN ranks as -inf)
+ *     n_b    = max{ n <= L_b : draft[cu_draft[b]+i] == t_i for all i < n }
+ *     bonus_b = t_{n_b}
+ * A draft id outside [0, vocab) never matches.  n_rows must equal
+ * cu_draft[n_branch] + n_branch.  row_argmax_d (nullable) receives every t_i.
+ * logits_d must be 16-byte aligned and row_stride_elems a multiple of 8.
+ * Calls that share a scratch buffer must not overlap on the device.
+ */
+int lr_accept_greedy(lr_ctx *ctx, const void *logits_d, int64_t row_stride_elems,
+                     const int32_t *draft_ids_d, const int32_t *cu_draft_d, int32_t n_branch, int32_t n_rows,
+                     int32_t *n_accept_d, int32_t *bonus_id_d, int32_t *row_argmax_d,
+                     void *scratch_d, void *stream);
+
+/*
+ * Step-level commit (Algorithm 1, last two lines: j* = index of the first
+ * rejected draft step, output = accepted draft steps followed by the decisive
+ * target step).  verdict_d: uint8 [sum_r gamma_r], request r's verdicts at
+ * req_span_off[r] - r.  Per request r:
+ *     n_steps_accepted = j*;  survivor = lowest-numbered branch of depth j*
+ *     (-1 if none);  kept_tail = own_len - L + n_accept of the survivor (0 if
+ *     none);  committed_len = prefix + segments 1..j* + kept_tail.
+ * keep list (CSR by request: keep_off [n_req+1], keep_pages / keep_valid sized
+ * n_page_slots): prefix pages, pages of segments 1..j*, the first
+ * ceil(kept_tail/16) tail pages of the survivor, each with its number of valid
+ * tokens.  free list (free_off, free_pages): pages of segments j*+1..gamma,
+ * then the branch tails in branch order (for the survivor only the pages past
+ * the kept ones).  keep and free together list every page slot of the request
+ * exactly once.  No KV data is moved.
+ */
+int lr_commit(lr_plan *plan, const uint8_t *verdict_d, const int32_t *n_accept_d,
+              int32_t *n_steps_accepted_d, int32_t *survivor_d, int32_t *committed_len_d,
+              int32_t *keep_off_d, int32_t *keep_pages_d, int32_t *keep_valid_d,
+              int32_t *free_off_d, int32_t *free_pages_d, void *stream);
+
+/* ---- whole pass with host buffers ---------------------------------------- */
+
+/* Host-side inputs and outputs of one pass; every pointer is a HOST pointer
+ * (pinned memory makes the copies asynchronous).  The KV pools stay on the
+ * device: they are the engine's resident cache, not a per-pass input. */
+typedef struct lr_pass_host_io {
+  const void *q_h;            /* [n_q_rows][n_q_heads][head_dim] bf16 */
+  const void *logits_h;       /* [n_rows][vocab] bf16, dense rows      */
+  const int32_t *draft_ids_h; /* [sum L_b]                             */
+  const uint8_t *verdict_h;   /* [sum gamma_r]                         */
+  void *out_h;                /* [n_q_rows][n_q_heads][head_dim] bf16  */
+  int32_t *n_accept_h, *bonus_id_h;                          /* [n_branch] */
+  int32_t *n_steps_accepted_h, *survivor_h, *committed_len_h; /* [n_req]   */
+  int32_t *keep_off_h, *free_off_h;                           /* [n_req+1] */
+  int32_t *keep_pages_h, *keep_valid_h, *free_pages_h;        /* [n_page_slots] */
+} lr_pass_host_io;
+
+/* Bytes of device staging lr_verify_pass_host needs for this plan. */
+int lr_pass_staging_bytes(const lr_plan *plan, size_t *bytes_out);
+
+/* One whole pass from host buffers: copies Q, logits, draft ids and verdicts to
+ * the device staging buffer, runs the three steps, copies every result back and
+ * WAITS for the stream.  staging_d: caller-owned device memory of
+ * lr_pass_staging_bytes, zero-filled before its first use.  Returns the device
+ * status like lr_poll_status. */
+int lr_verify_pass_host(lr_plan *plan, const lr_pass_host_io *io, const void *k_pool_d, const void *v_pool_d,
+                        void *staging_d, size_t staging_bytes, float softmax_scale, void *stream);
+
+/* ---- status ------------------------------------------------------------- */
+
+/* Waits for `stream`, reads the plan's device status word and clears it.
+ * Returns LR_OK, LR_ETIMEOUT or LR_EBOUNDS; *detail_out (nullable) receives a
+ * kernel-specific code saying where it happened. */
+int lr_poll_status(lr_plan *plan, void *stream, int32_t *detail_out);
+
+/* Number of kernels the library has launched on behalf of this context. */
+int64_t lr_launch_count(const lr_ctx *ctx);
+
+const char *lr_strerror(int status);
+const char *lr_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LR_VERIFY_H_ */

@@ -1,0 +1,209 @@
+// Greedy token-level acceptance: one streaming pass over the bf16 logits.
+//
+// Grid (chunks of a row, rows).  Each CTA reduces 8192 consecutive logits of
+// one row to (max value, lowest index), publishes it with one 64-bit atomicMax
+// on the row's key and takes a ticket; the CTA holding the last ticket turns the
+// row keys into n_accept / bonus per branch and zeroes the scratch again.
+//
+// The work is bound by HBM reads: 2 bytes per logit, read once, 16-byte loads,
+// four independent loads in flight per thread.  The maximum is taken with
+// packed bf16x2 max instructions on whole 16-byte vectors (about one
+// instruction per logit); the index is resolved only inside the winning vector.
+#include "lr_common.cuh"
+
+namespace lr {
+
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kVecPerThread = 4;                          // 16-byte vectors per thread per CTA
+constexpr int kChunk = kThreads * kVecPerThread * 8;      // logits per CTA
+
+// Monotone map of a float (already NaN-free, -0 folded to +0) to an unsigned key.
+__device__ __forceinline__ uint32_t order_key(float x) {
+  uint32_t u = __float_as_uint(x == 0.0f ? 0.0f : x);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+__device__ __forceinline__ uint4 ld_stream(const uint4 *p) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+               : "l"(p));
+  return v;
+}
+
+__device__ __forceinline__ __nv_bfloat162 as_bf2(uint32_t u) {
+  __nv_bfloat162 r;
+  *reinterpret_cast<uint32_t *>(&r) = u;
+  return r;
+}
+
+__device__ __forceinline__ float bf_lo(uint32_t u) { return __uint_as_float(u << 16); }
+__device__ __forceinline__ float bf_hi(uint32_t u) { return __uint_as_float(u & 0xFFFF0000u); }
+
+// NaN counts as -inf.
+__device__ __forceinline__ float denan(float x) { return (x != x) ? -INFINITY : x; }
+
+// max over the 8 bf16 of a vector; NaNs are ignored by the packed max (an all-NaN
+// vector gives NaN, which then fails every "greater than" test).
+__device__ __forceinline__ float vec_max(const uint4 &v) {
+  __nv_bfloat162 a = __hmax2(as_bf2(v.x), as_bf2(v.y));
+  __nv_bfloat162 b = __hmax2(as_bf2(v.z), as_bf2(v.w));
+  a = __hmax2(a, b);
+  uint32_t u = *reinterpret_cast<uint32_t *>(&a);
+  return fmaxf(bf_lo(u), bf_hi(u));
+}
+
+// index (0..7) of the first element of v equal to x (x is the vector's max, not NaN)
+__device__ __forceinline__ int first_equal(const uint4 &v, float x) {
+  const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+  int idx = 7;
+#pragma unroll
+  for (int i = 3; i >= 0; --i) {
+    if (bf_hi(w[i]) == x) idx = 2 * i + 1;
+    if (bf_lo(w[i]) == x) idx = 2 * i;
+  }
+  return idx;
+}
+
+struct Best {
+  float v;
+  int32_t i;
+};
+
+__device__ __forceinline__ Best better(Best a, Best b) {
+  // higher value wins; equal values: lower index wins
+  if (b.v > a.v || (b.v == a.v && b.i < a.i)) return b;
+  return a;
+}
+
+__global__ void __launch_bounds__(kThreads)
+accept_greedy_kernel(const uint16_t *__restrict__ logits, int64_t row_stride, int32_t vocab,
+                     const int32_t *__restrict__ draft_ids, const int32_t *__restrict__ cu_draft, int32_t n_branch,
+                     int32_t n_rows, int32_t *__restrict__ n_accept, int32_t *__restrict__ bonus_id,
+                     int32_t *__restrict__ row_argmax, unsigned long long *scratch) {
+  unsigned int *counter = reinterpret_cast<unsigned int *>(scratch);
+  unsigned long long *row_key = scratch + 1;
+  const int row = blockIdx.y;
+  const int tid = threadIdx.x;
+  const int64_t c0 = (int64_t)blockIdx.x * kChunk;
+  const uint16_t *rp = logits + (int64_t)row * row_stride;
+  const int32_t n_vec = vocab >> 3;  // whole 16-byte vectors in the row
+
+  // Per thread: vectors are visited in increasing index order and only a strictly
+  // greater maximum replaces the current one, so the earliest maximum is kept.
+  Best best;
+  best.v = -INFINITY;
+  best.i = 0x7FFFFFFF;  // "owns no element": loses every tie
+  {
+    const uint4 *vp = reinterpret_cast<const uint4 *>(rp);
+    uint4 v[kVecPerThread];
+    int32_t vi[kVecPerThread];
+#pragma unroll
+    for (int k = 0; k < kVecPerThread; ++k) {
+      vi[k] = (int32_t)(c0 >> 3) + k * kThreads + tid;
+      if (vi[k] < n_vec) v[k] = ld_stream(vp + vi[k]);
+    }
+    uint4 bv = make_uint4(0, 0, 0, 0);
+    int32_t bvi = -1;
+#pragma unroll
+    for (int k = 0; k < kVecPerThread; ++k) {
+      if (vi[k] < n_vec) {
+        float m = denan(vec_max(v[k]));
+        if (m > best.v || bvi < 0) {
+          best.v = m;
+          bv = v[k];
+          bvi = vi[k];
+        }
+      }
+    }
+    // a maximum of -inf means every element is -inf or NaN: the first one wins
+    if (bvi >= 0) best.i = bvi * 8 + (best.v == -INFINITY ? 0 : first_equal(bv, best.v));
+  }
+  // ragged end of the row (vocab not a multiple of 8): up to 7 single elements
+  if (blockIdx.x == gridDim.x - 1) {
+    int32_t e = n_vec * 8 + tid;
+    if (e < vocab) {
+      Best t;
+      t.v = denan(bf_lo((uint32_t)rp[e]));
+      t.i = e;
+      best = better(best, t);
+    }
+  }
+  // warp, then block reduction
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) {
+    Best o;
+    o.v = __shfl_down_sync(0xFFFFFFFFu, best.v, off);
+    o.i = __shfl_down_sync(0xFFFFFFFFu, best.i, off);
+    best = better(best, o);
+  }
+  __shared__ float s_v[kThreads / 32];
+  __shared__ int32_t s_i[kThreads / 32];
+  __shared__ int s_last;
+  if ((tid & 31) == 0) {
+    s_v[tid >> 5] = best.v;
+    s_i[tid >> 5] = best.i;
+  }
+  __syncthreads();
+  if (tid == 0) {
+    for (int w = 1; w < kThreads / 32; ++w) {
+      Best o;
+      o.v = s_v[w];
+      o.i = s_i[w];
+      best = better(best, o);
+    }
+    unsigned long long key = ((unsigned long long)order_key(best.v) << 32) | (unsigned long long)(0xFFFFFFFFu - (uint32_t)best.i);
+    atomicMax(row_key + row, key);
+    __threadfence();
+    unsigned int total = gridDim.x * gridDim.y;
+    unsigned int t = atomicAdd(counter, 1u);
+    s_last = (t == total - 1);
+  }
+  __syncthreads();
+  if (!s_last) return;
+
+  // ---- last CTA: per-branch longest matching prefix + bonus ------------------
+  __threadfence();
+  volatile unsigned long long *vk = row_key;
+  for (int b = tid; b < n_branch; b += kThreads) {
+    const int32_t d0 = cu_draft[b], L = cu_draft[b + 1] - d0;
+    const int32_t r0 = d0 + b;
+    int32_t n = 0;
+    while (n < L) {
+      int32_t t = (int32_t)(0xFFFFFFFFu - (uint32_t)(vk[r0 + n] & 0xFFFFFFFFull));
+      if (draft_ids[d0 + n] != t) break;
+      ++n;
+    }
+    n_accept[b] = n;
+    bonus_id[b] = (int32_t)(0xFFFFFFFFu - (uint32_t)(vk[r0 + n] & 0xFFFFFFFFull));
+  }
+  if (row_argmax != nullptr)
+    for (int r = tid; r < n_rows; r += kThreads)
+      row_argmax[r] = (int32_t)(0xFFFFFFFFu - (uint32_t)(vk[r] & 0xFFFFFFFFull));
+  __syncthreads();
+  for (int r = tid; r < n_rows; r += kThreads) row_key[r] = 0ull;
+  if (tid == 0) *counter = 0u;
+}
+
+}  // namespace
+
+int launch_accept(lr_ctx *ctx, const void *logits, int64_t stride, const int32_t *drafts, const int32_t *cu_draft,
+                  int32_t n_branch, int32_t n_rows, int32_t *n_accept, int32_t *bonus, int32_t *row_argmax,
+                  void *scratch, cudaStream_t s) {
+  const int32_t vocab = ctx->model.vocab;
+  const unsigned chunks = (unsigned)((vocab + kChunk - 1) / kChunk);
+  if (n_rows > 65535) {
+    set_error("lr_accept_greedy: more than 65535 logits rows in one call");
+    return LR_EUNSUPPORTED;
+  }
+  dim3 grid(chunks, (unsigned)n_rows);
+  accept_greedy_kernel<<<grid, kThreads, 0, s>>>(reinterpret_cast<const uint16_t *>(logits), stride, vocab, drafts,
+                                                  cu_draft, n_branch, n_rows, n_accept, bonus, row_argmax,
+                                                  reinterpret_cast<unsigned long long *>(scratch));
+  ctx->launches++;
+  return cuda_fail(cudaGetLastError(), "accept_greedy_kernel launch");
+}
+
+}  // namespace lr

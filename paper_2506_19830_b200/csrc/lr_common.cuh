@@ -1,0 +1,149 @@
+// Shared declarations of the verify-pass library: host objects, the device view
+// of a plan, and small device helpers.  Internal; the public surface is
+// include/lr_verify.h.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <stddef.h>
+
+#include <string.h>
+#include <string>
+#include <vector>
+
+#include "lr_verify.h"
+
+namespace lr {
+
+constexpr int kPage = 16;
+
+// Device status word layout: [0] = code (0 ok, 1 timeout, 2 bounds), [1] = detail.
+enum DevStatus : int { kDevOk = 0, kDevTimeout = 1, kDevBounds = 2 };
+
+// Device view of the integer tables of a batch (all pointers into the plan workspace).
+struct DevBatch {
+  const int32_t *req_span_off, *span_len, *span_slot;
+  const int32_t *br_req, *br_depth, *br_own_len, *br_own_slot, *br_n_draft;
+  const int32_t *cu_q, *cu_draft, *page_ids;
+  const int32_t *req_br_off;  // [n_req+1] branch range of each request
+  const int32_t *span_req;    // [n_span] owning request of each span
+  int32_t n_req, n_branch, n_span, n_page_slots, n_q_rows;
+  int32_t n_q_heads, n_kv_heads, head_dim, group;
+  int64_t n_pool_pages;
+  int32_t *status;  // [2]
+};
+
+// ---- tensor-core attention plan (device side) -------------------------------
+// A request's *extended chain* is the list of its page slots in the order
+// prefix, segments 1..gamma, branch tails; consecutive groups of 8 pages form
+// 128-key tiles.  An (request, kv head, M-group) triple is a *group*; its tiles
+// are cut into contiguous *pieces*, one or more per CTA.
+struct TcPage {      // one per extended-chain page
+  int32_t page;      // physical page id
+  uint32_t meta;     // bits 0-4 valid tokens (1..16), 5-12 min depth to see it, 13-20 owner branch (local, +1; 0 = chain), 21-31 first tail token index of the page / 16
+};
+struct TcPiece {
+  int32_t req, kv_head, mgroup;   // which rows x which KV head
+  int32_t tile_begin, tile_end;   // tiles of the request's extended chain
+  int32_t partial_slot;           // < 0: sole piece of its group, write final output directly
+  int32_t group_id;
+  int32_t pad;
+};
+struct TcReq {
+  int32_t page_off;     // first TcPage of the request
+  int32_t n_pages;      // extended-chain pages
+  int32_t q_row0, n_q;  // query token range of the request
+  int32_t br0, n_br;    // branch range
+  int32_t n_dense_tiles;  // leading tiles made only of full prefix pages (no masking needed)
+  int32_t pad;
+};
+struct TcGroup {
+  int32_t req, kv_head, mgroup;
+  int32_t partial_begin, n_partial;  // partial slots to merge (n_partial >= 2), else unused
+  int32_t pad[3];
+};
+struct DevTcPlan {
+  const TcPage *pages;
+  const TcPiece *pieces;
+  const int32_t *cta_piece_off;  // [n_cta+1]
+  const TcReq *reqs;
+  const TcGroup *groups;
+  int32_t n_cta, n_groups, n_merge_groups;
+  int32_t tokens_per_mtile;  // floor(128 / group)
+  float *partial_o;          // [n_partial_slots][256][head_dim] fp32, unnormalised
+  float *partial_ml;         // [n_partial_slots][256][2] (running max in log2 units, sum)
+  int32_t *tickets;          // [n_groups], zero between launches
+};
+
+}  // namespace lr
+
+struct lr_ctx {
+  lr_model model;
+  int device;
+  int sm_count;
+  int64_t launches;
+  void *tmap_encode;  // cuTensorMapEncodeTiled entry point (driver), resolved lazily
+  struct TmapEntry { const void *ptr; int64_t n_pages; alignas(64) unsigned char map[128]; };
+  std::vector<TmapEntry> tmaps;
+};
+
+struct lr_plan {
+  lr_ctx *ctx;
+  lr::DevBatch dev;
+  lr::DevTcPlan tc;
+  bool tc_ok;             // shape allows the tensor-core path
+  int attention_path;     // 0 auto, 1 generic, 2 tensor core
+  std::vector<unsigned char> staging;  // host copy of the uploaded image (kept alive for the async copy)
+  void *pinned;           // pinned host image
+  size_t image_bytes;
+  void *workspace_d;
+  size_t workspace_bytes;
+  // host copies needed at launch time
+  int32_t n_rows_logits, n_drafts, n_verdicts;
+  std::vector<int32_t> cu_draft_h;
+};
+
+namespace lr {
+
+// Byte image of everything lr_plan_create uploads; sections are 256-byte aligned.
+struct Image {
+  std::vector<unsigned char> bytes;
+  size_t add(const void *src, size_t n) {
+    size_t off = (bytes.size() + 255) / 256 * 256;
+    bytes.resize(off + n);
+    if (src && n) memcpy(bytes.data() + off, src, n);
+    return off;
+  }
+};
+
+// Host-side result of planning the tensor-core attention for one batch.
+struct TcHostPlan {
+  bool ok = false;  // shape supported by the tensor-core path
+  size_t o_pages = 0, o_pieces = 0, o_cta_piece_off = 0, o_reqs = 0, o_groups = 0;  // image offsets
+  int n_cta = 0, n_groups = 0, n_pieces = 0, n_partial_slots = 0, tokens_per_mtile = 0;
+  // scratch region behind the image: tickets (zeroed at plan creation), then (max, sum) pairs, then fp32 partial outputs
+  size_t s_tickets = 0, s_ml = 0, s_o = 0, scratch_bytes = 0, scratch_zero_bytes = 0;
+};
+int tc_build_host_plan(const lr_ctx *ctx, const lr_batch *b, const int32_t *req_br_off, TcHostPlan &out, Image &img);
+void tc_bind_device_plan(const TcHostPlan &h, unsigned char *image_base, unsigned char *scratch_base, lr_plan *p);
+
+void set_error(const char *fmt, ...);
+int cuda_fail(cudaError_t e, const char *what);
+
+// kernels (each file exposes launchers)
+int init_kernels(lr_ctx *ctx);  // per-device function attributes; called by lr_create
+int init_commit_kernel();
+int init_attn_tc_kernel();
+int launch_attn_generic(lr_plan *p, const void *q, const void *k, const void *v, void *out, float *lse, float scale,
+                        cudaStream_t s);
+int launch_attn_tc(lr_plan *p, const void *q, const void *k, const void *v, void *out, float *lse, float scale,
+                   cudaStream_t s);
+int launch_accept(lr_ctx *ctx, const void *logits, int64_t stride, const int32_t *drafts, const int32_t *cu_draft,
+                  int32_t n_branch, int32_t n_rows, int32_t *n_accept, int32_t *bonus, int32_t *row_argmax,
+                  void *scratch, cudaStream_t s);
+int launch_commit(lr_plan *p, const uint8_t *verdict, const int32_t *n_accept, int32_t *n_steps, int32_t *survivor,
+                  int32_t *committed, int32_t *keep_off, int32_t *keep_pages, int32_t *keep_valid, int32_t *free_off,
+                  int32_t *free_pages, cudaStream_t s);
+
+}  // namespace lr
