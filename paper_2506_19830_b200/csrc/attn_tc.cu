@@ -568,38 +568,62 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant_
 }
 
 // Merge of the split-KV partials of one group: O = sum_j 2^(m_j - M) O_j / sum_j 2^(m_j - M) l_j.
+// One warp per query row (grid: groups x 32 CTAs of 8 warps); the slots are read in a fixed order.
 __global__ void __launch_bounds__(256)
 attn_tc_merge_kernel(DevBatch d, DevTcPlan tc, uint16_t *__restrict__ out, float *__restrict__ lse) {
   const TcGroup g = tc.groups[blockIdx.x];
   const TcReq rq = tc.reqs[g.req];
   const int T = tc.tokens_per_mtile, G = d.group;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  for (int row = blockIdx.y * 8 + warp; row < 256; row += gridDim.y * 8) {
-    const int mt = 2 * g.mgroup + (row >> 7), r = row & 127;
-    const int tok = mt * T + r / G;
-    if (r >= T * G || tok >= rq.n_q) continue;
-    const int64_t qi = (int64_t)(rq.q_row0 + tok) * d.n_q_heads + g.kv_head * G + r % G;
-    float M = -INFINITY;
-    for (int j = 0; j < g.n_partial; ++j) M = fmaxf(M, tc.partial_ml[((int64_t)(g.partial_begin + j) * 256 + row) * 2]);
-    float L = 0.f;
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int j = 0; j < g.n_partial; ++j) {
-      const int64_t prow = (int64_t)(g.partial_begin + j) * 256 + row;
-      const float2 ml = *reinterpret_cast<const float2 *>(tc.partial_ml + prow * 2);
-      if (ml.y == 0.f) continue;  // this piece saw no key of the row
-      const float w = exp2f(ml.x - M);
-      L += w * ml.y;
-      const float4 o = *reinterpret_cast<const float4 *>(tc.partial_o + prow * kD + lane * 4);
-      acc.x += w * o.x;
-      acc.y += w * o.y;
-      acc.z += w * o.z;
-      acc.w += w * o.w;
+  const int row = blockIdx.y * 8 + warp;
+  const int mt = 2 * g.mgroup + (row >> 7), r = row & 127;
+  const int tok = mt * T + r / G;
+  if (r >= T * G || tok >= rq.n_q) return;
+  const int64_t qi = (int64_t)(rq.q_row0 + tok) * d.n_q_heads + g.kv_head * G + r % G;
+  const int64_t prow0 = (int64_t)g.partial_begin * 256 + row;
+  // lane j holds (m, l) of slot j, 32 slots at a time
+  float M = -INFINITY;
+  for (int j0 = 0; j0 < g.n_partial; j0 += 32) {
+    const int j = j0 + lane;
+    float mj = -INFINITY;
+    if (j < g.n_partial) {
+      const float2 ml = *reinterpret_cast<const float2 *>(tc.partial_ml + (prow0 + (int64_t)j * 256) * 2);
+      mj = ml.y > 0.f ? ml.x : -INFINITY;
     }
-    const float inv = 1.0f / L;
-    uint2 pk = make_uint2(pack_bf16(acc.x * inv, acc.y * inv), pack_bf16(acc.z * inv, acc.w * inv));
-    *reinterpret_cast<uint2 *>(out + qi * kD + lane * 4) = pk;
-    if (lse != nullptr && lane == 0) lse[qi] = (M + log2f(L)) * 0.6931471805599453f;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mj = fmaxf(mj, __shfl_xor_sync(0xFFFFFFFFu, mj, o));
+    M = fmaxf(M, mj);
   }
+  float L = 0.f;
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int j0 = 0; j0 < g.n_partial; j0 += 32) {
+    const int j = j0 + lane;
+    float wl = 0.f, w = 0.f;
+    if (j < g.n_partial) {
+      const float2 ml = *reinterpret_cast<const float2 *>(tc.partial_ml + (prow0 + (int64_t)j * 256) * 2);
+      if (ml.y > 0.f) {  // a piece that saw no key of the row contributes nothing
+        w = exp2f(ml.x - M);
+        wl = w * ml.y;
+      }
+    }
+    const int n = min(32, g.n_partial - j0);
+#pragma unroll 4
+    for (int jj = 0; jj < n; ++jj) {
+      const float wj = __shfl_sync(0xFFFFFFFFu, w, jj);
+      L += __shfl_sync(0xFFFFFFFFu, wl, jj);
+      const float4 o = *reinterpret_cast<const float4 *>(tc.partial_o + (prow0 + (int64_t)(j0 + jj) * 256) * kD + lane * 4);
+      if (wj != 0.f) {
+        acc.x = fmaf(wj, o.x, acc.x);
+        acc.y = fmaf(wj, o.y, acc.y);
+        acc.z = fmaf(wj, o.z, acc.z);
+        acc.w = fmaf(wj, o.w, acc.w);
+      }
+    }
+  }
+  const float inv = 1.0f / L;
+  uint2 pk = make_uint2(pack_bf16(acc.x * inv, acc.y * inv), pack_bf16(acc.z * inv, acc.w * inv));
+  *reinterpret_cast<uint2 *>(out + qi * kD + lane * 4) = pk;
+  if (lse != nullptr && lane == 0) lse[qi] = (M + log2f(L)) * 0.6931471805599453f;
 }
 
 // ---- tensor maps -------------------------------------------------------------------
@@ -807,7 +831,7 @@ int launch_attn_tc(lr_plan *p, const void *q, const void *k, const void *v, void
   p->ctx->launches++;
   if (int rc = cuda_fail(cudaGetLastError(), "attn_tc_kernel launch")) return rc;
   if (p->tc.n_merge_groups > 0) {
-    dim3 grid((unsigned)p->tc.n_merge_groups, 4);
+    dim3 grid((unsigned)p->tc.n_merge_groups, 32);
     attn_tc_merge_kernel<<<grid, 256, 0, s>>>(p->dev, p->tc, reinterpret_cast<uint16_t *>(out), lse);
     p->ctx->launches++;
     if (int rc = cuda_fail(cudaGetLastError(), "attn_tc_merge_kernel launch")) return rc;

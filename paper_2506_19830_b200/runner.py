@@ -30,7 +30,17 @@ class DeviceInputs:
         self.k_pool = bf16_tensor(tensors.k_pool, device)
         self.v_pool = bf16_tensor(tensors.v_pool, device)
         self.cu_draft = torch.from_numpy(np.ascontiguousarray(batch.cu_draft, dtype=np.int32)).to(device)
-        self.logits = bf16_tensor(tensors.logits, device) if with_logits and tensors.logits is not None else None
+        self.logits = None
+        if with_logits and tensors.logits is not None:
+            n_rows, vocab = tensors.logits.shape
+            stride = (vocab + 7) // 8 * 8  # the C ABI wants a row stride that is a multiple of 8 elements
+            if stride == vocab:
+                self.logits = bf16_tensor(tensors.logits, device)
+            else:
+                # padding columns hold +inf: they lie beyond `vocab` and must never be looked at
+                padded = np.full((n_rows, stride), 0x7F80, dtype=np.uint16)
+                padded[:, :vocab] = tensors.logits
+                self.logits = bf16_tensor(padded, device)[:, :vocab]
         self.draft_ids = (torch.from_numpy(np.ascontiguousarray(tensors.draft_ids, dtype=np.int32)).to(device)
                           if tensors.draft_ids is not None else None)
         v = tensors.verdict if tensors.verdict is not None and len(tensors.verdict) else np.zeros(1, dtype=np.uint8)
