@@ -52,7 +52,8 @@ constexpr int kTileBytes = 32768;  // [2 halves of 64 channels][128 keys or rows
 constexpr int kHalfBytes = 16384;
 constexpr int kThreads = 320;
 constexpr int kPagesPerTile = 8;
-constexpr uint32_t kSpinLimit = 1u << 22;
+constexpr uint64_t kWaitLimitNs = 1000ull * 1000ull * 1000ull;  // one second per wait, measured on the global timer
+constexpr uint64_t kDrainLimitNs = 50ull * 1000ull * 1000ull;
 constexpr float kRescaleThreshold = 8.0f;  // log2 units: P stays below 2^8
 
 struct __align__(8) Ctrl {
@@ -80,10 +81,10 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint64_t *bar, uint32_t parity
   uint32_t ok;
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
       "selp.b32 %0, 1, 0, p;\n\t}"
       : "=r"(ok)
-      : "r"(smem_u32(bar)), "r"(parity)
+      : "r"(smem_u32(bar)), "r"(parity), "r"(20000u)  // suspend for at most 20 us per try
       : "memory");
   return ok;
 }
@@ -180,11 +181,23 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return *reinterpret_cast<uint32_t *>(&t);
 }
 
-// Bounded wait.  Returns false when the wait expired or another role of the CTA gave up.
+__device__ __forceinline__ uint64_t global_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+
+// Bounded wait: gives up after kWaitLimitNs of wall time.  Returns false when the wait expired or
+// another role of the CTA gave up.
 __device__ __forceinline__ bool wait_bar(uint64_t *bar, uint32_t parity, Ctrl *ctrl, int32_t *status, int code) {
-  for (uint32_t i = 0; i < kSpinLimit; ++i) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const uint64_t t0 = global_ns();
+  for (uint32_t i = 1;; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
-    if ((i & 255u) == 255u && *reinterpret_cast<volatile int *>(&ctrl->abort_flag)) return false;
+    if ((i & 31u) == 0u) {
+      if (*reinterpret_cast<volatile int *>(&ctrl->abort_flag)) return false;
+      if (global_ns() - t0 > kWaitLimitNs) break;
+    }
   }
   *reinterpret_cast<volatile int *>(&ctrl->abort_flag) = 1;
   status[0] = kDevTimeout;
@@ -304,8 +317,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant_
       // give the copies already in flight a bounded time to land before the CTA exits
       for (uint32_t back = 1; back <= (uint32_t)kStages && back <= it; ++back) {
         const uint32_t j = it - back;
-        for (uint32_t i = 0; i < (1u << 16); ++i)
-          if (mbar_try_wait(&ctrl->kv_full[j % kStages], (j / kStages) & 1u)) break;
+        const uint64_t t0 = global_ns();
+        while (!mbar_try_wait(&ctrl->kv_full[j % kStages], (j / kStages) & 1u))
+          if (global_ns() - t0 > kDrainLimitNs) break;
       }
     }
   } else if (warp == 1) {
@@ -410,8 +424,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant_
     if (!ok && lane == 0) {
       // let every MMA already issued retire before tensor memory is released
       tc_commit(&ctrl->drain);
-      for (uint32_t i = 0; i < (1u << 20); ++i)
-        if (mbar_try_wait(&ctrl->drain, 0)) break;
+      const uint64_t t0 = global_ns();
+      while (!mbar_try_wait(&ctrl->drain, 0))
+        if (global_ns() - t0 > kDrainLimitNs) break;
     }
     __syncwarp();
   } else {
