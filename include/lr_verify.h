@@ -177,6 +177,33 @@ int lr_accept_greedy(lr_ctx *ctx, const void *logits_d, int64_t row_stride_elems
                      void *scratch_d, void *stream);
 
 /*
+ * lr_accept_greedy without a caller-provided scratch buffer.  (The paper has no
+ * counterpart: this is a packaging variant of the call above, same results.)
+ *
+ * For callers that cannot obtain device memory at the point of the call: a
+ * serving engine that handed every free byte of HBM to its KV cache at start-up,
+ * or code running where cudaMalloc is off limits because it synchronises the
+ * whole device and may fail late.  The row keys and the ticket counter live in
+ * an array built into the library (8 * (LR_ACCEPT_STATIC_MAX_ROWS + 1) bytes on
+ * every GPU that loads it, held until the process exits).  The call allocates
+ * nothing, neither with cudaMalloc nor through any library.
+ *
+ *   - n_rows > LR_ACCEPT_STATIC_MAX_ROWS is rejected with LR_EINVAL.
+ *   - The first call on a device looks up the array's device address (a
+ *     cudaGetSymbolAddress call, made with ctx's device current); make that
+ *     first call outside any stream capture.
+ *   - All calls on one device share the one array.  Each call clears the part
+ *     it uses on `stream` before its kernel runs, so leftovers of an earlier
+ *     call never matter, but two calls whose device work overlaps in time
+ *     (different streams, no dependency between them) race on it.
+ * Arguments, results and errors are otherwise those of lr_accept_greedy.
+ */
+#define LR_ACCEPT_STATIC_MAX_ROWS 4096
+int lr_accept_greedy_static(lr_ctx *ctx, const void *logits_d, int64_t row_stride_elems,
+                            const int32_t *draft_ids_d, const int32_t *cu_draft_d, int32_t n_branch, int32_t n_rows,
+                            int32_t *n_accept_d, int32_t *bonus_id_d, int32_t *row_argmax_d, void *stream);
+
+/*
  * Step-level commit (Algorithm 1, last two lines: j* = index of the first
  * rejected draft step, output = accepted draft steps followed by the decisive
  * target step).  verdict_d: uint8 [sum_r gamma_r], request r's verdicts at

@@ -21,6 +21,7 @@ STATUS_NAMES = {0: "LR_OK", -1: "LR_EINVAL", -2: "LR_EUNSUPPORTED", -3: "LR_ECUD
                 -6: "LR_ENOMEM"}
 
 PATH_AUTO, PATH_GENERIC, PATH_TENSOR_CORE = 0, 1, 2
+ACCEPT_STATIC_MAX_ROWS = 4096  # LR_ACCEPT_STATIC_MAX_ROWS
 
 
 class LrError(RuntimeError):
@@ -74,6 +75,7 @@ def lib() -> C.CDLL:
             "lr_verify_attention": [vp, vp, vp, vp, vp, vp, f32, vp],
             "lr_accept_scratch_bytes": [i32, C.POINTER(sz)],
             "lr_accept_greedy": [vp, vp, i64, vp, vp, i32, i32, vp, vp, vp, vp, vp],
+            "lr_accept_greedy_static": [vp, vp, i64, vp, vp, i32, i32, vp, vp, vp, vp],
             "lr_commit": [vp] + [vp] * 10 + [vp],
             "lr_pass_staging_bytes": [vp, C.POINTER(sz)],
             "lr_verify_pass_host": [vp, C.POINTER(lr_pass_host_io), vp, vp, vp, sz, f32, vp],
@@ -175,6 +177,16 @@ class Context:
         _check(lib().lr_accept_greedy(self.handle, _ptr(logits), logits.stride(0), _ptr(draft_ids), _ptr(cu_draft), n_branch,
                                       n_rows, _ptr(n_accept), _ptr(bonus_id), _ptr(row_argmax), _ptr(scratch),
                                       _stream_ptr(stream)), "lr_accept_greedy")
+
+    def lr_accept_greedy_static(self, logits: torch.Tensor, draft_ids: torch.Tensor, cu_draft: torch.Tensor,
+                                n_accept: torch.Tensor, bonus_id: torch.Tensor, row_argmax: Optional[torch.Tensor] = None,
+                                stream=None) -> None:
+        """``lr_accept_greedy`` on the scratch array built into the library: no scratch argument and no
+        device allocation; at most ``ACCEPT_STATIC_MAX_ROWS`` logits rows."""
+        n_branch = cu_draft.numel() - 1
+        _check(lib().lr_accept_greedy_static(self.handle, _ptr(logits), logits.stride(0), _ptr(draft_ids), _ptr(cu_draft),
+                                             n_branch, logits.shape[0], _ptr(n_accept), _ptr(bonus_id), _ptr(row_argmax),
+                                             _stream_ptr(stream)), "lr_accept_greedy_static")
 
     @staticmethod
     def accept_scratch(n_rows: int, device) -> torch.Tensor:

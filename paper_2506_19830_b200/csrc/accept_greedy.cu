@@ -187,7 +187,39 @@ accept_greedy_kernel(const uint16_t *__restrict__ logits, int64_t row_stride, in
   if (tid == 0) *counter = 0u;
 }
 
+// Scratch of lr_accept_greedy_static: row keys + ticket counter for up to LR_ACCEPT_STATIC_MAX_ROWS rows.
+// Lives in every context that loads the library, for the life of the process.
+static __device__ __align__(256) unsigned long long g_static_scratch[LR_ACCEPT_STATIC_MAX_ROWS + 1];
+
 }  // namespace
+
+// Device address of g_static_scratch per device ordinal, resolved on the first call for that device.
+static void *g_static_scratch_addr[64] = {nullptr};
+
+int launch_accept_static(lr_ctx *ctx, const void *logits, int64_t stride, const int32_t *drafts, const int32_t *cu_draft,
+                         int32_t n_branch, int32_t n_rows, int32_t *n_accept, int32_t *bonus, int32_t *row_argmax,
+                         cudaStream_t s) {
+  if (n_rows > LR_ACCEPT_STATIC_MAX_ROWS) {
+    set_error("lr_accept_greedy_static: %d logits rows, the built-in scratch holds at most %d; use lr_accept_greedy",
+              n_rows, LR_ACCEPT_STATIC_MAX_ROWS);
+    return LR_EINVAL;
+  }
+  if (ctx->device < 0 || ctx->device >= 64) {
+    set_error("lr_accept_greedy_static: device ordinal %d not supported", ctx->device);
+    return LR_EUNSUPPORTED;
+  }
+  if (int rc = cuda_fail(cudaSetDevice(ctx->device), "cudaSetDevice")) return rc;
+  void *ptr = g_static_scratch_addr[ctx->device];
+  if (ptr == nullptr) {
+    // In host code the array's name is only a handle; the kernel needs the address the symbol has
+    // on *this* device.  Done once per device, with that device current.
+    if (int rc = cuda_fail(cudaGetSymbolAddress(&ptr, g_static_scratch), "cudaGetSymbolAddress(static scratch)")) return rc;
+    g_static_scratch_addr[ctx->device] = ptr;
+  }
+  // Every call shares the array and it keeps what the last call left: start from zero regardless.
+  if (int rc = cuda_fail(cudaMemsetAsync(ptr, 0, 8 * ((size_t)n_rows + 1), s), "cudaMemsetAsync(static scratch)")) return rc;
+  return launch_accept(ctx, logits, stride, drafts, cu_draft, n_branch, n_rows, n_accept, bonus, row_argmax, ptr, s);
+}
 
 int launch_accept(lr_ctx *ctx, const void *logits, int64_t stride, const int32_t *drafts, const int32_t *cu_draft,
                   int32_t n_branch, int32_t n_rows, int32_t *n_accept, int32_t *bonus, int32_t *row_argmax,

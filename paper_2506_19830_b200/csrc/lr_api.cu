@@ -368,6 +368,26 @@ extern "C" int lr_accept_greedy(lr_ctx *ctx, const void *logits, int64_t stride,
                        reinterpret_cast<cudaStream_t>(stream));
 }
 
+extern "C" int lr_accept_greedy_static(lr_ctx *ctx, const void *logits, int64_t stride, const int32_t *drafts,
+                                       const int32_t *cu_draft, int32_t n_branch, int32_t n_rows, int32_t *n_accept,
+                                       int32_t *bonus, int32_t *row_argmax, void *stream) {
+  if (!ctx || !logits || !cu_draft || !n_accept || !bonus || (!drafts && n_rows > n_branch)) {
+    set_error("lr_accept_greedy_static: null argument");
+    return LR_EINVAL;
+  }
+  if (n_branch < 0 || n_rows < n_branch) {
+    set_error("lr_accept_greedy_static: n_rows %d < n_branch %d", n_rows, n_branch);
+    return LR_EINVAL;
+  }
+  if (((uintptr_t)logits & 15) != 0 || (stride & 7) != 0 || stride < ctx->model.vocab) {
+    set_error("lr_accept_greedy_static: logits must be 16-byte aligned with a row stride that is a multiple of 8 and >= vocab");
+    return LR_EINVAL;
+  }
+  if (n_branch == 0) return LR_OK;
+  return launch_accept_static(ctx, logits, stride, drafts, cu_draft, n_branch, n_rows, n_accept, bonus, row_argmax,
+                              reinterpret_cast<cudaStream_t>(stream));
+}
+
 extern "C" int lr_commit(lr_plan *p, const uint8_t *verdict, const int32_t *n_accept, int32_t *n_steps, int32_t *survivor,
                          int32_t *committed, int32_t *keep_off, int32_t *keep_pages, int32_t *keep_valid,
                          int32_t *free_off, int32_t *free_pages, void *stream) {
