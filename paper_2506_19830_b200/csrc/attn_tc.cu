@@ -6,27 +6,40 @@
 // head -- (query token, head-in-group) pairs, floor(128/G) tokens per 128-row
 // M-tile -- are processed against a tile at once, so a KV page is fetched from
 // HBM once for every branch and every GQA head that can see it.  A *group* is
-// (request, KV head, pair of M-tiles); the tiles of all groups, weighted, are
-// cut into equal contiguous ranges, one per CTA (one CTA per SM).  A range may
-// cover parts of several groups (*pieces*).  A piece that is a whole group
-// writes bf16 output directly; otherwise it writes an fp32 partial (running
-// max, sum, unnormalised O) and a small second kernel merges the partials of a
-// group in a fixed order.
+// (request, KV head, one or two M-tiles); the tiles of all groups, weighted, are
+// cut into equal contiguous ranges, one per CTA (one CTA per SM); a range may
+// cover parts of several groups (*pieces*).
 //
-// One CTA = 10 warps:
-//   warp 0      TMA producer: per tile 16 + 16 bulk tensor copies (one per page
-//               and 64-channel half, K then V) into a 4-stage ring of 32 KB
-//               buffers in the 128-byte-swizzled layout the MMA descriptors read.
-//   warp 1      MMA issuer: tcgen05.mma (M=128, N=128, K=16, bf16 -> fp32) for
-//               S = Q K^T (both operands in shared memory) and O += P V (P read
-//               from tensor memory, V from shared memory as the N-major operand).
-//   warps 2-5   softmax of M-tile 0, one thread per query row (tcgen05.ld gives
-//   warps 6-9   softmax of M-tile 1  a thread its whole row, so row max and row
-//               sum need no cross-lane traffic): visibility masks, running max
-//               with lazy rescaling of O in tensor memory, exp2, bf16 P written
-//               back over S.
-// Tensor memory (512 columns): S0 | S1 | O0 | O1, 128 fp32 columns each; P_m
-// occupies the first 64 columns of S_m.
+// A CTA runs two independent *streams*, each with its own score tile S, output
+// accumulator O (both in tensor memory), MMA issuer warp and softmax warpgroup:
+// for a piece with two M-tiles stream s is M-tile s over every tile; for a piece
+// with one M-tile stream s takes every other tile (a split of the keys inside
+// the CTA).  While one stream is in its softmax the tensor pipe works for the
+// other.  A stream whose result is the only contribution to its M-tile writes
+// bf16 output; otherwise it writes an fp32 partial (reference exponent, sum,
+// unnormalised O) and a small second kernel merges the partials of an M-tile in
+// a fixed order.
+//
+// One CTA = 11 warps:
+//   warp 0      TMA producer: the Q tiles of a piece (3-D boxes: 64 channels x G
+//               heads x T tokens, so that the rows land packed) and, per tile,
+//               16 + 16 bulk tensor copies (one per page and 64-channel half, K
+//               and V) into a 5-stage ring of 32 KB buffers, all in the
+//               128-byte-swizzled layout the MMA descriptors read.  No multicast.
+//   warps 1, 2  MMA issuers of stream 0 and 1: tcgen05.mma (M=128, N=128, K=16,
+//               bf16 -> fp32) for S = Q K^T (both operands in shared memory) and
+//               O += P V (P read from tensor memory, V from shared memory as the
+//               N-major operand).  Issue blocks while the tensor pipe is full, so
+//               one issuer per stream lets the waits of one overlap the MMAs of
+//               the other.
+//   warps 3-6   softmax of stream 0, one thread per query row: tcgen05.ld gives a
+//   warps 7-10  softmax of stream 1  thread its whole row of S in registers, so
+//               row max and row sum need no cross-lane traffic.  One sweep:
+//               max (3-input max), lazy rescale of O in tensor memory only when
+//               the maximum grew by more than 2^8, exp2 with packed fp32 FMA/ADD,
+//               bf16 P written back over S.
+// Tensor memory (512 columns): S0 | S1 | O0 | O1, 128 fp32 columns each; P_s
+// occupies the first 64 columns of S_s.
 //
 // Visibility.  Tiles made only of full prefix pages need no mask.  In every other
 // tile each page carries (valid tokens, minimum depth, owning branch, tail
@@ -35,10 +48,12 @@
 // invalid token slots are zeroed in shared memory before the PV product so that
 // whatever the slack holds (NaN included) cannot reach the output.
 //
-// Every wait on an mbarrier is bounded; when one expires the CTA raises its abort
-// flag, records LR_ETIMEOUT in the status word, drains what it has in flight,
-// frees its tensor memory and returns.
+// Every wait on an mbarrier is bounded by the global timer; when one expires the
+// CTA raises its abort flag, records LR_ETIMEOUT in the status word, drains what
+// it has in flight, frees its tensor memory and returns.
 #include <cuda.h>
+
+#include <algorithm>
 
 #include "lr_common.cuh"
 
@@ -47,10 +62,10 @@ namespace lr {
 namespace {
 
 constexpr int kD = 128;
-constexpr int kStages = 4;
+constexpr int kStages = 5;
 constexpr int kTileBytes = 32768;  // [2 halves of 64 channels][128 keys or rows][128 B]
 constexpr int kHalfBytes = 16384;
-constexpr int kThreads = 320;
+constexpr int kThreads = 352;
 constexpr int kPagesPerTile = 8;
 constexpr uint64_t kWaitLimitNs = 1000ull * 1000ull * 1000ull;  // one second per wait, measured on the global timer
 constexpr uint64_t kDrainLimitNs = 50ull * 1000ull * 1000ull;
@@ -58,12 +73,13 @@ constexpr float kRescaleThreshold = 8.0f;  // log2 units: P stays below 2^8
 
 struct __align__(8) Ctrl {
   uint64_t kv_full[kStages], kv_empty[kStages];
+  uint64_t q_full, q_empty;
   uint64_t s_full[2], p_full[2], o_done[2];
-  uint64_t q_full[2], piece_done[2], drain;
+  uint64_t epi_done, stagger, drain[2];
   uint32_t tmem_base;
   int abort_flag;
 };
-constexpr int kSmemBytes = 1024 + 2 * kTileBytes + kStages * kTileBytes + 1024;
+constexpr int kSmemBytes = 2 * kTileBytes + kStages * kTileBytes + 1024;  // tiles, then Ctrl; the base must be 1024-aligned
 
 // ---- PTX wrappers ----------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -88,6 +104,17 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint64_t *bar, uint32_t parity
       : "memory");
   return ok;
 }
+__device__ __forceinline__ uint32_t mbar_test_wait(uint64_t *bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.b32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok;
+}
 __device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -99,11 +126,17 @@ __device__ __forceinline__ void tc_commit(uint64_t *bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 
-// 2-D tiled bulk tensor copy global -> shared, completion on an mbarrier (no multicast).
+// Tiled bulk tensor copies global -> shared, completion on an mbarrier (no multicast).
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int32_t x, int32_t y, uint64_t *bar) {
   asm volatile(
       "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(dst),
       "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, int32_t x, int32_t y, int32_t z, uint64_t *bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];" ::"r"(dst),
+      "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y), "r"(z)
       : "memory");
 }
 
@@ -131,50 +164,50 @@ __device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_
       : "memory");
 }
 
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
-  uint32_t r[32];
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
-        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
-        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-      : "r"(taddr)
-      : "memory");
-  tc_wait_ld();
-#pragma unroll
-  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+// tcgen05.ld / tcgen05.st, shape 32x32b: thread i of the warp owns lane (base + i), consecutive columns.
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+               : "r"(taddr)
+               : "memory");
 }
-__device__ __forceinline__ void tmem_st32(uint32_t taddr, const float (&v)[32]) {
-  asm volatile(
-      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
-      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
-      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};" ::"r"(taddr),
-      "r"(__float_as_uint(v[0])), "r"(__float_as_uint(v[1])), "r"(__float_as_uint(v[2])), "r"(__float_as_uint(v[3])),
-      "r"(__float_as_uint(v[4])), "r"(__float_as_uint(v[5])), "r"(__float_as_uint(v[6])), "r"(__float_as_uint(v[7])),
-      "r"(__float_as_uint(v[8])), "r"(__float_as_uint(v[9])), "r"(__float_as_uint(v[10])), "r"(__float_as_uint(v[11])),
-      "r"(__float_as_uint(v[12])), "r"(__float_as_uint(v[13])), "r"(__float_as_uint(v[14])), "r"(__float_as_uint(v[15])),
-      "r"(__float_as_uint(v[16])), "r"(__float_as_uint(v[17])), "r"(__float_as_uint(v[18])), "r"(__float_as_uint(v[19])),
-      "r"(__float_as_uint(v[20])), "r"(__float_as_uint(v[21])), "r"(__float_as_uint(v[22])), "r"(__float_as_uint(v[23])),
-      "r"(__float_as_uint(v[24])), "r"(__float_as_uint(v[25])), "r"(__float_as_uint(v[26])), "r"(__float_as_uint(v[27])),
-      "r"(__float_as_uint(v[28])), "r"(__float_as_uint(v[29])), "r"(__float_as_uint(v[30])), "r"(__float_as_uint(v[31]))
-      : "memory");
+__device__ __forceinline__ void tmem_ld64(uint32_t taddr, uint32_t (&r)[64]) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x64.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32, %33, %34, %35, %36, %37, %38, %39, %40, %41, %42, %43, %44, %45, %46, %47, %48, %49, %50, %51, %52, %53, %54, %55, %56, %57, %58, %59, %60, %61, %62, %63}, [%64];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31]), "=r"(r[32]), "=r"(r[33]), "=r"(r[34]), "=r"(r[35]), "=r"(r[36]), "=r"(r[37]), "=r"(r[38]), "=r"(r[39]), "=r"(r[40]), "=r"(r[41]), "=r"(r[42]), "=r"(r[43]), "=r"(r[44]), "=r"(r[45]), "=r"(r[46]), "=r"(r[47]), "=r"(r[48]), "=r"(r[49]), "=r"(r[50]), "=r"(r[51]), "=r"(r[52]), "=r"(r[53]), "=r"(r[54]), "=r"(r[55]), "=r"(r[56]), "=r"(r[57]), "=r"(r[58]), "=r"(r[59]), "=r"(r[60]), "=r"(r[61]), "=r"(r[62]), "=r"(r[63])
+               : "r"(taddr)
+               : "memory");
 }
-__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
-  asm volatile(
-      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
-      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};" ::"r"(taddr),
-      "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
-      "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
-      : "memory");
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};" ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+               : "memory");
 }
 
 __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+// packed fp32 pairs: d = a * b + c and d = a + b on both halves with one instruction each
+__device__ __forceinline__ float2 ffma2(float2 a, float2 b, float2 c) {
+  float2 d;
+  asm("{\n\t.reg .b64 ra, rb, rc, rd;\n\tmov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\tmov.b64 rc, {%6, %7};\n\t"
+      "fma.rn.f32x2 rd, ra, rb, rc;\n\tmov.b64 {%0, %1}, rd;\n\t}"
+      : "=f"(d.x), "=f"(d.y)
+      : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y), "f"(c.x), "f"(c.y));
+  return d;
+}
+__device__ __forceinline__ float2 fadd2(float2 a, float2 b) {
+  float2 d;
+  asm("{\n\t.reg .b64 ra, rb, rd;\n\tmov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\t"
+      "add.rn.f32x2 rd, ra, rb;\n\tmov.b64 {%0, %1}, rd;\n\t}"
+      : "=f"(d.x), "=f"(d.y)
+      : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
+  return d;
 }
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
@@ -190,7 +223,7 @@ __device__ __forceinline__ uint64_t global_ns() {
 // Bounded wait: gives up after kWaitLimitNs of wall time.  Returns false when the wait expired or
 // another role of the CTA gave up.
 __device__ __forceinline__ bool wait_bar(uint64_t *bar, uint32_t parity, Ctrl *ctrl, int32_t *status, int code) {
-  if (mbar_try_wait(bar, parity)) return true;
+  if (mbar_test_wait(bar, parity)) return true;
   const uint64_t t0 = global_ns();
   for (uint32_t i = 1;; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
@@ -205,6 +238,28 @@ __device__ __forceinline__ bool wait_bar(uint64_t *bar, uint32_t parity, Ctrl *c
   return false;
 }
 
+// ---- ring order ----------------------------------------------------------------------
+// Within a piece of n tiles the producer emits K and V tiles in the order the MMA issuers first
+// touch them.  With la = K tiles issued ahead of the first PV (1 for two M-tiles, 2 for the
+// even/odd split): K(0..min(la,n)-1), then for u = 0..n-1: V(u), and K(u+la) while u+la < n.
+struct RingOrder {
+  int n, la, la_c, np;  // np = number of (V, K) pairs
+  __device__ __forceinline__ RingOrder(int n_, int mode) : n(n_), la(mode == 2 ? 1 : 2) {
+    la_c = min(la, n);
+    np = max(0, n - la);
+  }
+  __device__ __forceinline__ int pos_k(int t) const { return t < la ? t : la_c + 2 * (t - la) + 1; }
+  __device__ __forceinline__ int pos_v(int u) const { return u < np ? la_c + 2 * u : la_c + 2 * np + (u - np); }
+  // step i (= ring position within the piece) of the 2n steps -> tile, and whether it is a V tile
+  __device__ __forceinline__ int step(int i, bool &is_v) const {
+    if (i < la_c) { is_v = false; return i; }
+    const int j = i - la_c;
+    if (j < 2 * np) { is_v = !(j & 1); return (j >> 1) + ((j & 1) ? la : 0); }
+    is_v = true;
+    return np + (j - 2 * np);
+  }
+};
+
 struct RowInfo {
   int depth;       // segments the row sees; -1 for padding rows
   int branch;      // local branch index within the request; -1 for padding rows
@@ -212,8 +267,8 @@ struct RowInfo {
   int64_t q_index; // (query row * n_q_heads + head), -1 for padding rows
 };
 
-// Row r (0..127) of M-tile mt of a group: token mt*T + r/G, head kv*G + r%G.
-__device__ __forceinline__ RowInfo row_info(const DevBatch &d, const TcReq &rq, int T, int mt, int r, int kv) {
+// Row r (0..127) of M-tile mt of (request, KV head): token mt*T + r/G, head kv*G + r%G.
+__device__ __forceinline__ RowInfo row_info(const DevBatch &d, const DevTcPlan &tc, const TcReq &rq, int T, int mt, int r, int kv) {
   RowInfo ri;
   ri.depth = -1;
   ri.branch = -1;
@@ -223,12 +278,10 @@ __device__ __forceinline__ RowInfo row_info(const DevBatch &d, const TcReq &rq, 
   const int tok = mt * T + r / G;
   if (r < T * G && tok < rq.n_q) {
     const int row = rq.q_row0 + tok;
-    int b = rq.br0;
-    while (b + 1 < rq.br0 + rq.n_br && d.cu_q[b + 1] <= row) ++b;
-    const int i = row - d.cu_q[b], q_len = d.cu_q[b + 1] - d.cu_q[b];
-    ri.depth = d.br_depth[b];
-    ri.branch = b - rq.br0;
-    ri.limit = d.br_own_len[b] - q_len + i;
+    const int2 w = __ldg(reinterpret_cast<const int2 *>(tc.rows + row));
+    ri.depth = w.x & 0xFFFF;
+    ri.branch = w.x >> 16;
+    ri.limit = w.y;
     ri.q_index = (int64_t)row * d.n_q_heads + kv * G + r % G;
   }
   return ri;
@@ -242,29 +295,87 @@ __device__ __forceinline__ int page_n_ok(uint32_t meta, const RowInfo &ri) {
   return max(n, 0);
 }
 
+__device__ __forceinline__ float bits_f(uint32_t u) { return __uint_as_float(u); }
+
+// -inf on the score columns of one 64-key half that the row does not see
+__device__ __forceinline__ void mask_half(uint32_t (&v)[64], const int *n_ok) {
+#pragma unroll
+  for (int p = 0; p < 4; ++p) {
+    const int n = n_ok[p];
+    if (n < kPage) {
+#pragma unroll
+      for (int c = 0; c < kPage; ++c)
+        if (c >= n) v[p * kPage + c] = 0xFF800000u;
+    }
+  }
+}
+__device__ __forceinline__ float max_half(const uint32_t (&v)[64]) {
+  float a = -INFINITY, b = -INFINITY, c = -INFINITY, e = -INFINITY;
+#pragma unroll
+  for (int i = 0; i < 64; i += 8) {
+    a = max3(a, bits_f(v[i]), bits_f(v[i + 1]));
+    b = max3(b, bits_f(v[i + 2]), bits_f(v[i + 3]));
+    c = max3(c, bits_f(v[i + 4]), bits_f(v[i + 5]));
+    e = max3(e, bits_f(v[i + 6]), bits_f(v[i + 7]));
+  }
+  return fmaxf(fmaxf(a, b), fmaxf(c, e));
+}
+// P = exp2(scale * s - m) for 64 scores -> 32 packed bf16 pairs; returns the fp32 sum
+__device__ __forceinline__ float exp_half(const uint32_t (&v)[64], uint32_t (&pk)[32], float scale_log2, float neg_m) {
+  const float2 sc = make_float2(scale_log2, scale_log2), nm = make_float2(neg_m, neg_m);
+  float2 acc0 = make_float2(0.f, 0.f), acc1 = make_float2(0.f, 0.f);
+#pragma unroll
+  for (int i = 0; i < 64; i += 4) {
+    float2 y0 = ffma2(make_float2(bits_f(v[i]), bits_f(v[i + 1])), sc, nm);
+    float2 y1 = ffma2(make_float2(bits_f(v[i + 2]), bits_f(v[i + 3])), sc, nm);
+    y0.x = ex2(y0.x);
+    y0.y = ex2(y0.y);
+    y1.x = ex2(y1.x);
+    y1.y = ex2(y1.y);
+    acc0 = fadd2(acc0, y0);
+    acc1 = fadd2(acc1, y1);
+    pk[i >> 1] = pack_bf16(y0.x, y0.y);
+    pk[(i >> 1) + 1] = pack_bf16(y1.x, y1.y);
+  }
+  acc0 = fadd2(acc0, acc1);
+  return acc0.x + acc0.y;
+}
+
 __global__ void __launch_bounds__(kThreads, 1)
-attn_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map, DevBatch d, DevTcPlan tc,
-               const uint16_t *__restrict__ q, uint16_t *__restrict__ out, float *__restrict__ lse, float scale_log2) {
-  extern __shared__ unsigned char smem_raw[];
-  unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+attn_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map,
+               const __grid_constant__ CUtensorMap q_map, DevBatch d, DevTcPlan tc, uint16_t *__restrict__ out,
+               float *__restrict__ lse, float scale_log2) {
+  extern __shared__ __align__(1024) unsigned char smem[];
+  if ((smem_u32(smem) & 1023u) != 0u) {  // the swizzled tiles need a 1024-byte aligned base
+    if (threadIdx.x == 0) {
+      d.status[0] = kDevBounds;
+      d.status[1] = 250;
+    }
+    return;
+  }
   unsigned char *q_smem = smem;                         // 2 x 32 KB
   unsigned char *kv_smem = smem + 2 * kTileBytes;       // kStages x 32 KB
   Ctrl *ctrl = reinterpret_cast<Ctrl *>(kv_smem + kStages * kTileBytes);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
+  // rows of a Q tile that no copy writes must hold finite values
+  for (int i = threadIdx.x; i < 2 * kTileBytes / 16; i += kThreads) reinterpret_cast<uint4 *>(q_smem)[i] = make_uint4(0, 0, 0, 0);
+  fence_proxy_async();
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
       mbar_init(&ctrl->kv_full[s], 1);
-      mbar_init(&ctrl->kv_empty[s], 1);
+      mbar_init(&ctrl->kv_empty[s], 2);  // one arrival per MMA issuer
     }
-    for (int m = 0; m < 2; ++m) {
-      mbar_init(&ctrl->s_full[m], 1);
-      mbar_init(&ctrl->p_full[m], 128);
-      mbar_init(&ctrl->o_done[m], 1);
-      mbar_init(&ctrl->q_full[m], 128);
-      mbar_init(&ctrl->piece_done[m], 128);
+    mbar_init(&ctrl->q_full, 1);
+    mbar_init(&ctrl->q_empty, 2);
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(&ctrl->s_full[s], 1);
+      mbar_init(&ctrl->p_full[s], 128);
+      mbar_init(&ctrl->o_done[s], 1);
+      mbar_init(&ctrl->drain[s], 1);
     }
-    mbar_init(&ctrl->drain, 1);
+    mbar_init(&ctrl->epi_done, 256);
+    mbar_init(&ctrl->stagger, 128);
     ctrl->abort_flag = 0;
     fence_barrier_init();
   }
@@ -277,105 +388,160 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant_
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *reinterpret_cast<volatile uint32_t *>(&ctrl->tmem_base);
+  // inputs may come from the kernel launched just before this one
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
   const int piece0 = tc.cta_piece_off[blockIdx.x], piece1 = tc.cta_piece_off[blockIdx.x + 1];
   const int T = tc.tokens_per_mtile;
+  const int G = d.group;
 
   if (warp == 0) {
     // ======================= TMA producer ==========================================
-    uint32_t it = 0;
+    uint32_t ring = 0, q_count = 0;
     bool ok = true;
+    const uint32_t q_box_bytes = (uint32_t)(64 * G * T * 2);
     for (int pc = piece0; pc < piece1 && ok; ++pc) {
       const TcPiece pi = tc.pieces[pc];
       const TcReq rq = tc.reqs[pi.req];
-      for (int t = pi.tile_begin; t < pi.tile_end && ok; ++t) {
-        const int npages = min(kPagesPerTile, rq.n_pages - t * kPagesPerTile);
-        int64_t page = 0;
-        if (lane < 16 && (lane >> 1) < npages) {
-          page = tc.pages[rq.page_off + t * kPagesPerTile + (lane >> 1)].page;
-          if (page < 0 || page >= d.n_pool_pages) {  // never fetch outside the pool
+      const int n = pi.tile_end - pi.tile_begin;
+      // Q tiles of the piece, once the MMAs of the previous piece no longer read the buffers
+      ok = wait_bar(&ctrl->q_empty, (q_count & 1u) ^ 1u, ctrl, d.status, 205);
+      if (!ok) break;
+      if (lane == 0) mbar_arrive_expect_tx(&ctrl->q_full, (uint32_t)pi.n_mt * 2u * q_box_bytes);
+      __syncwarp();
+      if (lane < 2 * pi.n_mt)
+        tma_load_3d(smem_u32(q_smem) + (lane >> 1) * kTileBytes + (lane & 1) * kHalfBytes, &q_map, (lane & 1) * 64, pi.kv_head * G,
+                    rq.q_row0 + (pi.mtile0 + (lane >> 1)) * T, &ctrl->q_full);
+      ++q_count;
+      const RingOrder ord(n, pi.n_mt);
+      // Page ids arrive 32 at a time (one per lane = 4 tiles) and one chunk ahead of their first use,
+      // so no step of the loop waits for a load it has just issued.
+      auto load_chunk = [&](int c) -> int32_t {
+        const int idx = c * 32 + lane;
+        int32_t pg = -1;  // absent page
+        if (idx < rq.n_pages) {
+          pg = tc.pages[rq.page_off + idx].page;
+          if (pg < 0 || pg >= d.n_pool_pages) {  // never fetch outside the pool
             d.status[0] = kDevBounds;
             d.status[1] = 200;
-            page = 0;
+            pg = 0;
           }
         }
-        for (int op = 0; op < 2 && ok; ++op, ++it) {
-          const uint32_t stage = it % kStages;
-          ok = wait_bar(&ctrl->kv_empty[stage], ((it / kStages) & 1u) ^ 1u, ctrl, d.status, 210);
-          if (!ok) break;
-          if (lane == 0) mbar_arrive_expect_tx(&ctrl->kv_full[stage], (uint32_t)npages * 4096u);
-          __syncwarp();
-          if (lane < 16 && (lane >> 1) < npages) {
-            const uint32_t dst = smem_u32(kv_smem + stage * kTileBytes) + (lane & 1) * kHalfBytes + (lane >> 1) * 2048;
-            tma_load_2d(dst, op == 0 ? &k_map : &v_map, (lane & 1) * 64, (int32_t)((page * d.n_kv_heads + pi.kv_head) * kPage),
-                        &ctrl->kv_full[stage]);
-          }
+        return pg;
+      };
+      int c_cur = pi.tile_begin >> 2;
+      int32_t pg_cur = load_chunk(c_cur), pg_nxt = load_chunk(c_cur + 1);
+      for (int i = 0; i < 2 * n && ok; ++i, ++ring) {
+        bool is_v;
+        const int t = pi.tile_begin + ord.step(i, is_v);
+        if (is_v && (t >> 2) > c_cur) {  // the V index is the oldest tile still needed
+          ++c_cur;
+          pg_cur = pg_nxt;
+          pg_nxt = load_chunk(c_cur + 1);
+        }
+        const int32_t page = __shfl_sync(0xFFFFFFFFu, (t >> 2) == c_cur ? pg_cur : pg_nxt, (t & 3) * 8 + ((lane & 15) >> 1));
+        const int npages = min(kPagesPerTile, rq.n_pages - t * kPagesPerTile);
+        const uint32_t stage = ring % kStages;
+        ok = wait_bar(&ctrl->kv_empty[stage], ((ring / kStages) & 1u) ^ 1u, ctrl, d.status, 210);
+        if (!ok) break;
+        if (lane == 0) mbar_arrive_expect_tx(&ctrl->kv_full[stage], (uint32_t)npages * 4096u);
+        __syncwarp();
+        if (lane < 16 && page >= 0) {
+          const uint32_t dst = smem_u32(kv_smem + stage * kTileBytes) + (lane & 1) * kHalfBytes + (lane >> 1) * 2048;
+          tma_load_2d(dst, is_v ? &v_map : &k_map, (lane & 1) * 64, (int32_t)(((int64_t)page * d.n_kv_heads + pi.kv_head) * kPage),
+                      &ctrl->kv_full[stage]);
         }
       }
     }
     if (!ok) {
       // give the copies already in flight a bounded time to land before the CTA exits
-      for (uint32_t back = 1; back <= (uint32_t)kStages && back <= it; ++back) {
-        const uint32_t j = it - back;
+      for (uint32_t back = 1; back <= (uint32_t)kStages && back <= ring; ++back) {
+        const uint32_t j = ring - back;
         const uint64_t t0 = global_ns();
         while (!mbar_try_wait(&ctrl->kv_full[j % kStages], (j / kStages) & 1u))
           if (global_ns() - t0 > kDrainLimitNs) break;
       }
     }
-  } else if (warp == 1) {
-    // ======================= MMA issuer =============================================
-    uint32_t it = 0, q_phase[2] = {0, 0}, done_phase[2] = {0, 0}, p_phase[2] = {0, 0};
+  } else if (warp <= 2) {
+    // ======================= MMA issuer of stream s ====================================
+    // Both issuers walk every ring position of a piece in order: a position this stream uses is
+    // consumed by its MMAs (released by a tcgen05.commit), one it does not use (the other
+    // stream's tiles in the even/odd split) is released with a plain arrive once it has landed.
+    // So neither issuer nor the producer can get a whole ring ahead of the other.
+    const int s = warp - 1;
+    uint32_t ring_base = 0, waited = 0, p_cnt = 0, pc_idx = 0;
     bool ok = true;
     const uint32_t q_addr = smem_u32(q_smem), kv_addr = smem_u32(kv_smem);
-    auto issue_qk = [&](int m, uint32_t stage) {
-      const uint32_t a = q_addr + m * kTileBytes, b = kv_addr + stage * kTileBytes;
+    const uint32_t s_tmem = tmem + s * 128, o_tmem = tmem + 256 + s * 128;
+    // Descriptors differ from a base only in the start-address field (units of 16 bytes).
+    const uint64_t qdesc0 = make_desc(q_addr, 16, 1024), kdesc0 = make_desc(kv_addr, 16, 1024),
+                   vdesc0 = make_desc(kv_addr, kHalfBytes, 1024);
+    auto issue_qk = [&](int m, uint32_t stage) {  // S_s = Q_m K^T
+      const uint64_t a = qdesc0 + (uint64_t)(m * (kTileBytes >> 4)), b = kdesc0 + (uint64_t)(stage * (kTileBytes >> 4));
 #pragma unroll
       for (int h = 0; h < 2; ++h)
 #pragma unroll
         for (int kk = 0; kk < 4; ++kk)
-          mma_ss(tmem + m * 128, make_desc(a + h * kHalfBytes + kk * 32, 16, 1024),
-                 make_desc(b + h * kHalfBytes + kk * 32, 16, 1024), kIdescQK, (h | kk) != 0);
+          mma_ss(s_tmem, a + (uint64_t)(h * (kHalfBytes >> 4) + kk * 2), b + (uint64_t)(h * (kHalfBytes >> 4) + kk * 2), kIdescQK,
+                 (h | kk) != 0);
     };
-    auto issue_pv = [&](int m, uint32_t stage, bool acc) {
-      const uint32_t b = kv_addr + stage * kTileBytes;
+    auto issue_pv = [&](uint32_t stage, bool acc) {  // O_s (+)= P_s V
+      const uint64_t b = vdesc0 + (uint64_t)(stage * (kTileBytes >> 4));
 #pragma unroll
-      for (int ks = 0; ks < 8; ++ks)
-        mma_ts(tmem + 256 + m * 128, tmem + m * 128 + ks * 8, make_desc(b + ks * 2048, kHalfBytes, 1024), kIdescPV,
-               acc || ks != 0);
+      for (int ks = 0; ks < 8; ++ks) mma_ts(o_tmem, s_tmem + ks * 8, b + (uint64_t)(ks * (2048 >> 4)), kIdescPV, acc || ks != 0);
     };
-    for (int pc = piece0; pc < piece1 && ok; ++pc) {
+    for (int pc = piece0; pc < piece1 && ok; ++pc, ++pc_idx) {
       const TcPiece pi = tc.pieces[pc];
       const TcReq rq = tc.reqs[pi.req];
-      const int n_mt = min(2, (rq.n_q + T - 1) / T - 2 * pi.mgroup);
-      for (int m = 0; m < n_mt && ok; ++m) {
-        ok = wait_bar(&ctrl->q_full[m], q_phase[m], ctrl, d.status, 220);
-        q_phase[m] ^= 1;
-      }
-      if (!ok) break;
-      tc_fence_after();
-      uint32_t sK = it % kStages;
-      ok = wait_bar(&ctrl->kv_full[sK], (it / kStages) & 1u, ctrl, d.status, 221);
-      ++it;
-      if (!ok) break;
-      tc_fence_after();
-      if (lane == 0) {
-        for (int m = 0; m < n_mt; ++m) {
-          issue_qk(m, sK);
-          tc_commit(&ctrl->s_full[m]);
+      const int n = pi.tile_end - pi.tile_begin, mode = pi.n_mt;
+      const RingOrder ord(n, mode);
+      const int my_units = mode == 2 ? n : (n - s + 1) / 2;
+      const int m_tile = mode == 2 ? s : 0;
+      // waits, in ring order, until absolute ring position `pos` has landed; positions on the way
+      // belong to the other stream and are released here
+      auto need = [&](uint32_t pos, int code) -> bool {
+        while (waited <= pos) {
+          if (!wait_bar(&ctrl->kv_full[waited % kStages], (waited / kStages) & 1u, ctrl, d.status, code)) return false;
+          if (waited < pos && lane == 0) mbar_arrive(&ctrl->kv_empty[waited % kStages]);
+          ++waited;
         }
-        tc_commit(&ctrl->kv_empty[sK]);
-      }
-      __syncwarp();
-      for (int t = pi.tile_begin; t < pi.tile_end && ok; ++t) {
-        const uint32_t sV = it % kStages;
-        ok = wait_bar(&ctrl->kv_full[sV], (it / kStages) & 1u, ctrl, d.status, 222);
-        ++it;
+        return true;
+      };
+      // after the MMAs that read the stage: arrives when they retire (the other issuer arrives for itself)
+      auto release = [&](uint32_t pos) { tc_commit(&ctrl->kv_empty[pos % kStages]); };
+      ok = wait_bar(&ctrl->q_full, pc_idx & 1u, ctrl, d.status, 220);
+      if (!ok) break;
+      if (my_units > 0) {
+        if (s == 1) {
+          // Start half a period behind stream 0 (after its first softmax), so that the two streams use
+          // the MUFU and the tensor pipe in turns instead of both at once.
+          ok = wait_bar(&ctrl->stagger, pc_idx & 1u, ctrl, d.status, 219);
+          if (!ok) break;
+        }
+        const uint32_t pos = ring_base + ord.pos_k(mode == 2 ? 0 : s);
+        ok = need(pos, 221);
         if (!ok) break;
-        if (t >= rq.n_dense_tiles) {
-          // zero the V rows of token slots that hold no valid token (slack of a last page, absent pages)
+        tc_fence_after();
+        if (lane == 0) {
+          issue_qk(m_tile, pos % kStages);
+          tc_commit(&ctrl->s_full[s]);
+          release(pos);
+        }
+        __syncwarp();
+      }
+      for (int j = 0; j < my_units && ok; ++j) {
+        const int t = mode == 2 ? j : 2 * j + s;
+        const uint32_t pos_v = ring_base + ord.pos_v(t), sV = pos_v % kStages;
+        ok = need(pos_v, 222);
+        if (!ok) break;
+        if (pi.tile_begin + t >= rq.n_dense_tiles) {
+          // zero the V rows of token slots that hold no valid token (slack of a last page, absent pages);
+          // with two M-tiles both issuers write the same zeros
           unsigned char *vs = kv_smem + sV * kTileBytes;
+          const TcPage *pg = tc.pages + rq.page_off + (pi.tile_begin + t) * kPagesPerTile;
           for (int p = 0; p < kPagesPerTile; ++p) {
-            const int valid = tc.pages[rq.page_off + t * kPagesPerTile + p].meta & 31;
+            const int valid = pg[p].meta & 31;
             for (int idx = lane; idx < (kPage - valid) * 16; idx += 32) {
               const int key = p * kPage + valid + (idx >> 4), h = (idx >> 3) & 1, ch = idx & 7;
               *reinterpret_cast<uint4 *>(vs + h * kHalfBytes + key * 128 + ch * 16) = make_uint4(0, 0, 0, 0);
@@ -384,111 +550,92 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant_
           fence_proxy_async();
           __syncwarp();
         }
-        const bool has_next = t + 1 < pi.tile_end;
+        const bool has_next = j + 1 < my_units;
+        uint32_t pos_k = 0;
         if (has_next) {
-          sK = it % kStages;
-          ok = wait_bar(&ctrl->kv_full[sK], (it / kStages) & 1u, ctrl, d.status, 223);
-          ++it;
+          pos_k = ring_base + ord.pos_k(mode == 2 ? j + 1 : 2 * (j + 1) + s);
+          ok = need(pos_k, 226);
           if (!ok) break;
         }
-        tc_fence_after();
-        for (int m = 0; m < n_mt && ok; ++m) {
-          ok = wait_bar(&ctrl->p_full[m], p_phase[m], ctrl, d.status, 224 + m);
-          p_phase[m] ^= 1;
+        if (j == 0 && pc_idx > 0) {  // the epilogue of the previous piece has read O_0 and O_1
+          ok = wait_bar(&ctrl->epi_done, (pc_idx - 1) & 1u, ctrl, d.status, 223);
           if (!ok) break;
-          tc_fence_after();
-          if (lane == 0) {
-            issue_pv(m, sV, t > pi.tile_begin);
-            tc_commit(&ctrl->o_done[m]);
-            if (has_next) {
-              issue_qk(m, sK);
-              tc_commit(&ctrl->s_full[m]);
-            }
-          }
-          __syncwarp();
         }
+        ok = wait_bar(&ctrl->p_full[s], p_cnt & 1u, ctrl, d.status, 224 + s);
+        ++p_cnt;
         if (!ok) break;
+        tc_fence_after();
         if (lane == 0) {
-          tc_commit(&ctrl->kv_empty[sV]);
-          if (has_next) tc_commit(&ctrl->kv_empty[sK]);
+          issue_pv(sV, j > 0);
+          tc_commit(&ctrl->o_done[s]);
+          release(pos_v);
+          if (has_next) {
+            issue_qk(m_tile, pos_k % kStages);
+            tc_commit(&ctrl->s_full[s]);
+            release(pos_k);
+          }
         }
         __syncwarp();
       }
       if (!ok) break;
-      for (int m = 0; m < n_mt && ok; ++m) {
-        ok = wait_bar(&ctrl->piece_done[m], done_phase[m], ctrl, d.status, 228);
-        done_phase[m] ^= 1;
+      // positions of the piece this stream never touched (the tail of the other stream's tiles)
+      ring_base += 2u * (uint32_t)n;
+      if (waited < ring_base) {
+        ok = need(ring_base - 1, 227);
+        if (!ok) break;
+        if (lane == 0) mbar_arrive(&ctrl->kv_empty[(ring_base - 1) % kStages]);
       }
-      tc_fence_after();
+      if (lane == 0) tc_commit(&ctrl->q_empty);  // every MMA of this stream retired: its reads of the Q buffers are done
+      __syncwarp();
     }
     if (!ok && lane == 0) {
       // let every MMA already issued retire before tensor memory is released
-      tc_commit(&ctrl->drain);
+      tc_commit(&ctrl->drain[s]);
       const uint64_t t0 = global_ns();
-      while (!mbar_try_wait(&ctrl->drain, 0))
+      while (!mbar_try_wait(&ctrl->drain[s], 0))
         if (global_ns() - t0 > kDrainLimitNs) break;
     }
     __syncwarp();
   } else {
     // ======================= softmax warpgroups ======================================
-    const int m = (warp - 2) >> 2;                 // M-tile within the pair
+    const int s = (warp - 3) >> 2;                 // stream
     const int quarter = warp & 3;                  // tensor-memory lane quarter this warp may access
     const int r = quarter * 32 + lane;             // row within the M-tile
     const uint32_t lane_base = tmem + ((uint32_t)(quarter * 32) << 16);
-    const uint32_t s_addr = lane_base + m * 128, o_addr = lane_base + 256 + m * 128;
-    uint32_t s_phase = 0, o_count = 0;
+    const uint32_t s_addr = lane_base + s * 128, o_addr = lane_base + 256 + s * 128;
+    uint32_t s_cnt = 0, o_cnt = 0;
     bool ok = true;
-    for (int pc = piece0; pc < piece1 && ok; ++pc) {
+    for (int pc = piece0; pc < piece1; ++pc) {
       const TcPiece pi = tc.pieces[pc];
       const TcReq rq = tc.reqs[pi.req];
-      const int n_mt = min(2, (rq.n_q + T - 1) / T - 2 * pi.mgroup);
-      if (m >= n_mt) continue;  // this M-tile does not exist in the piece
-      RowInfo ri = row_info(d, rq, T, 2 * pi.mgroup + m, r, pi.kv_head);
-      {
-        // stage this row of Q: 16 chunks of 16 B into the swizzled K-major layout
-        unsigned char *qs = q_smem + m * kTileBytes;
-        const uint4 *src = reinterpret_cast<const uint4 *>(q + ri.q_index * kD);
-#pragma unroll
-        for (int c = 0; c < 16; ++c) {
-          uint4 v = make_uint4(0, 0, 0, 0);
-          if (ri.q_index >= 0) v = __ldg(src + c);
-          *reinterpret_cast<uint4 *>(qs + (c >> 3) * kHalfBytes + r * 128 + (((c & 7) ^ (r & 7)) << 4)) = v;
-        }
-        fence_proxy_async();
-      }
-      mbar_arrive(&ctrl->q_full[m]);
-      float m_used = -INFINITY, l = 0.f;
-      {
-        for (int t = pi.tile_begin; t < pi.tile_end; ++t) {
-          ok = wait_bar(&ctrl->s_full[m], s_phase, ctrl, d.status, 230 + m);
-          s_phase ^= 1;
+      const int n = pi.tile_end - pi.tile_begin, mode = pi.n_mt;
+      const int my_units = mode == 2 ? n : (n - s + 1) / 2;
+      if (ok && my_units > 0) {
+        const RowInfo ri = row_info(d, tc, rq, T, mode == 2 ? pi.mtile0 + s : pi.mtile0, r, pi.kv_head);
+        float m_used = -INFINITY, l = 0.f;
+        for (int j = 0; j < my_units; ++j) {
+          const int t = pi.tile_begin + (mode == 2 ? j : 2 * j + s);
+          ok = wait_bar(&ctrl->s_full[s], s_cnt & 1u, ctrl, d.status, 230 + s);
+          ++s_cnt;
           if (!ok) break;
           tc_fence_after();
-          const bool masked = t >= rq.n_dense_tiles;
-          int n_ok[kPagesPerTile];
-          if (masked) {
+          uint32_t va[64], vb[64];
+          tmem_ld64(s_addr, va);
+          tmem_ld64(s_addr + 64, vb);
+          tc_wait_ld();
+          if (t >= rq.n_dense_tiles) {
+            int n_ok[kPagesPerTile];
             const uint4 *mp = reinterpret_cast<const uint4 *>(tc.pages + rq.page_off + t * kPagesPerTile);
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              const uint4 w = __ldg(mp + j);
-              n_ok[2 * j] = page_n_ok(w.y, ri);
-              n_ok[2 * j + 1] = page_n_ok(w.w, ri);
+            for (int jj = 0; jj < 4; ++jj) {
+              const uint4 w = __ldg(mp + jj);
+              n_ok[2 * jj] = page_n_ok(w.y, ri);
+              n_ok[2 * jj + 1] = page_n_ok(w.w, ri);
             }
+            mask_half(va, n_ok);
+            mask_half(vb, n_ok + 4);
           }
-          // pass 1: row maximum
-          float mx = -INFINITY;
-#pragma unroll
-          for (int ch = 0; ch < 4; ++ch) {
-            float v[32];
-            tmem_ld32(s_addr + ch * 32, v);
-#pragma unroll
-            for (int c = 0; c < 32; ++c) {
-              float x = v[c];
-              if (masked && (c & 15) >= n_ok[2 * ch + (c >> 4)]) x = -INFINITY;
-              mx = fmaxf(mx, x);
-            }
-          }
-          mx *= scale_log2;
+          const float mx = fmaxf(max_half(va), max_half(vb)) * scale_log2;
           // lazy rescale: only when the maximum grew by more than the threshold
           const bool grow = mx > m_used + kRescaleThreshold;
           if (__any_sync(0xFFFFFFFFu, grow)) {
@@ -497,72 +644,67 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant_
               l *= alpha;
               m_used = mx;
             }
-            if (t > pi.tile_begin) {
+            if (j > 0) {  // the PV product of this stream's previous unit has retired (its commit precedes s_full's)
 #pragma unroll
               for (int ch = 0; ch < 4; ++ch) {
-                float v[32];
-                tmem_ld32(o_addr + ch * 32, v);
+                uint32_t o[32];
+                tmem_ld32(o_addr + ch * 32, o);
+                tc_wait_ld();
 #pragma unroll
-                for (int c = 0; c < 32; ++c) v[c] *= alpha;
-                tmem_st32(o_addr + ch * 32, v);
+                for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(bits_f(o[c]) * alpha);
+                tmem_st32(o_addr + ch * 32, o);
               }
               tc_wait_st();
             }
           }
           const float neg_m = (m_used == -INFINITY) ? 0.f : -m_used;
-          // pass 2: P = exp2(scale * s - m), row sum, bf16 P over the first half of S
-#pragma unroll
-          for (int ch = 0; ch < 4; ++ch) {
-            float v[32];
-            tmem_ld32(s_addr + ch * 32, v);
-            uint32_t pk[16];
-#pragma unroll
-            for (int c = 0; c < 32; c += 2) {
-              float x0 = v[c], x1 = v[c + 1];
-              if (masked && (c & 15) >= n_ok[2 * ch + (c >> 4)]) x0 = -INFINITY;
-              if (masked && ((c + 1) & 15) >= n_ok[2 * ch + ((c + 1) >> 4)]) x1 = -INFINITY;
-              const float p0 = ex2(fmaf(x0, scale_log2, neg_m)), p1 = ex2(fmaf(x1, scale_log2, neg_m));
-              l += p0 + p1;
-              pk[c >> 1] = pack_bf16(p0, p1);
-            }
-            tmem_st16(s_addr + ch * 16, pk);
-          }
+          uint32_t pk[32];
+          l += exp_half(va, pk, scale_log2, neg_m);
+          tmem_st32(s_addr, pk);
+          l += exp_half(vb, pk, scale_log2, neg_m);
+          tmem_st32(s_addr + 32, pk);
           tc_wait_st();
           tc_fence_before();
-          mbar_arrive(&ctrl->p_full[m]);
+          mbar_arrive(&ctrl->p_full[s]);
+          if (s == 0 && j == 0) mbar_arrive(&ctrl->stagger);
         }
         if (ok) {
-          // epilogue: wait for the last PV of this piece, then normalise and store
-          o_count += (uint32_t)(pi.tile_end - pi.tile_begin);
-          ok = wait_bar(&ctrl->o_done[m], (o_count - 1) & 1u, ctrl, d.status, 240 + m);
+          // epilogue: wait for the last PV of this stream, then normalise and store
+          o_cnt += (uint32_t)my_units;
+          ok = wait_bar(&ctrl->o_done[s], (o_cnt - 1) & 1u, ctrl, d.status, 240 + s);
         }
         if (ok) {
           tc_fence_after();
-          if (pi.partial_slot < 0) {
+          const int slot = pi.slot[s];
+          if (slot < 0) {
             const float inv = 1.0f / l;
 #pragma unroll
-            for (int ch = 0; ch < 4; ++ch) {
-              float v[32];
-              tmem_ld32(o_addr + ch * 32, v);
+            for (int hf = 0; hf < 2; ++hf) {
+              uint32_t o[64];
+              tmem_ld64(o_addr + hf * 64, o);
+              tc_wait_ld();
               if (ri.q_index >= 0) {
-                uint4 *dst = reinterpret_cast<uint4 *>(out + ri.q_index * kD + ch * 32);
+                uint4 *dst = reinterpret_cast<uint4 *>(out + ri.q_index * kD + hf * 64);
 #pragma unroll
-                for (int j = 0; j < 4; ++j)
-                  dst[j] = make_uint4(pack_bf16(v[8 * j] * inv, v[8 * j + 1] * inv), pack_bf16(v[8 * j + 2] * inv, v[8 * j + 3] * inv),
-                                      pack_bf16(v[8 * j + 4] * inv, v[8 * j + 5] * inv), pack_bf16(v[8 * j + 6] * inv, v[8 * j + 7] * inv));
+                for (int jj = 0; jj < 8; ++jj)
+                  dst[jj] = make_uint4(pack_bf16(bits_f(o[8 * jj]) * inv, bits_f(o[8 * jj + 1]) * inv),
+                                       pack_bf16(bits_f(o[8 * jj + 2]) * inv, bits_f(o[8 * jj + 3]) * inv),
+                                       pack_bf16(bits_f(o[8 * jj + 4]) * inv, bits_f(o[8 * jj + 5]) * inv),
+                                       pack_bf16(bits_f(o[8 * jj + 6]) * inv, bits_f(o[8 * jj + 7]) * inv));
               }
             }
             if (lse != nullptr && ri.q_index >= 0) lse[ri.q_index] = (m_used + log2f(l)) * 0.6931471805599453f;
           } else {
-            const int64_t prow = (int64_t)pi.partial_slot * 256 + m * 128 + r;
+            const int64_t prow = (int64_t)slot * 128 + r;
 #pragma unroll
-            for (int ch = 0; ch < 4; ++ch) {
-              float v[32];
-              tmem_ld32(o_addr + ch * 32, v);
+            for (int hf = 0; hf < 2; ++hf) {
+              uint32_t o[64];
+              tmem_ld64(o_addr + hf * 64, o);
+              tc_wait_ld();
               if (ri.q_index >= 0) {
-                float4 *dst = reinterpret_cast<float4 *>(tc.partial_o + prow * kD + ch * 32);
+                uint4 *dst = reinterpret_cast<uint4 *>(tc.partial_o + prow * kD + hf * 64);
 #pragma unroll
-                for (int j = 0; j < 8; ++j) dst[j] = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+                for (int jj = 0; jj < 16; ++jj) dst[jj] = make_uint4(o[4 * jj], o[4 * jj + 1], o[4 * jj + 2], o[4 * jj + 3]);
               }
             }
             if (ri.q_index >= 0) *reinterpret_cast<float2 *>(tc.partial_ml + prow * 2) = make_float2(m_used, l);
@@ -570,7 +712,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant_
           tc_fence_before();
         }
       }
-      mbar_arrive(&ctrl->piece_done[m]);
+      mbar_arrive(&ctrl->epi_done);
     }
   }
 
@@ -582,57 +724,64 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant_
   }
 }
 
-// Merge of the split-KV partials of one group: O = sum_j 2^(m_j - M) O_j / sum_j 2^(m_j - M) l_j.
-// One warp per query row (grid: groups x 32 CTAs of 8 warps); the slots are read in a fixed order.
+// Merge of the partials of one M-tile: O = sum_j 2^(m_j - M) O_j / sum_j 2^(m_j - M) l_j.
+// One warp per query row (grid: targets x 16 CTAs of 8 warps); the slots are read in a fixed order.
 __global__ void __launch_bounds__(256)
 attn_tc_merge_kernel(DevBatch d, DevTcPlan tc, uint16_t *__restrict__ out, float *__restrict__ lse) {
-  const TcGroup g = tc.groups[blockIdx.x];
+  const TcTarget g = tc.targets[blockIdx.x];
   const TcReq rq = tc.reqs[g.req];
   const int T = tc.tokens_per_mtile, G = d.group;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int row = blockIdx.y * 8 + warp;
-  const int mt = 2 * g.mgroup + (row >> 7), r = row & 127;
-  const int tok = mt * T + r / G;
-  if (r >= T * G || tok >= rq.n_q) return;
+  const int r = blockIdx.y * 8 + warp;
+  const int tok = g.mtile * T + r / G;
+  const bool live = r < T * G && tok < rq.n_q;
+  // the partials come from the kernel launched just before this one
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (!live) return;
   const int64_t qi = (int64_t)(rq.q_row0 + tok) * d.n_q_heads + g.kv_head * G + r % G;
-  const int64_t prow0 = (int64_t)g.partial_begin * 256 + row;
-  // lane j holds (m, l) of slot j, 32 slots at a time
-  float M = -INFINITY;
-  for (int j0 = 0; j0 < g.n_partial; j0 += 32) {
-    const int j = j0 + lane;
-    float mj = -INFINITY;
-    if (j < g.n_partial) {
-      const float2 ml = *reinterpret_cast<const float2 *>(tc.partial_ml + (prow0 + (int64_t)j * 256) * 2);
-      mj = ml.y > 0.f ? ml.x : -INFINITY;
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) mj = fmaxf(mj, __shfl_xor_sync(0xFFFFFFFFu, mj, o));
-    M = fmaxf(M, mj);
-  }
-  float L = 0.f;
+  const int64_t prow0 = (int64_t)g.slot_begin * 128 + r;
+  float M = -INFINITY, L = 0.f;
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-  for (int j0 = 0; j0 < g.n_partial; j0 += 32) {
+  for (int j0 = 0; j0 < g.n_slots; j0 += 32) {
+    // lane j holds (m, l) of slot j0 + j
     const int j = j0 + lane;
-    float wl = 0.f, w = 0.f;
-    if (j < g.n_partial) {
-      const float2 ml = *reinterpret_cast<const float2 *>(tc.partial_ml + (prow0 + (int64_t)j * 256) * 2);
-      if (ml.y > 0.f) {  // a piece that saw no key of the row contributes nothing
-        w = exp2f(ml.x - M);
-        wl = w * ml.y;
+    float mj = -INFINITY, lj = 0.f;
+    if (j < g.n_slots) {
+      const float2 ml = *reinterpret_cast<const float2 *>(tc.partial_ml + (prow0 + (int64_t)j * 128) * 2);
+      if (ml.y > 0.f) {  // a stream that saw no key of the row contributes nothing
+        mj = ml.x;
+        lj = ml.y;
       }
     }
-    const int n = min(32, g.n_partial - j0);
-#pragma unroll 4
-    for (int jj = 0; jj < n; ++jj) {
-      const float wj = __shfl_sync(0xFFFFFFFFu, w, jj);
-      L += __shfl_sync(0xFFFFFFFFu, wl, jj);
-      const float4 o = *reinterpret_cast<const float4 *>(tc.partial_o + (prow0 + (int64_t)(j0 + jj) * 256) * kD + lane * 4);
-      if (wj != 0.f) {
-        acc.x = fmaf(wj, o.x, acc.x);
-        acc.y = fmaf(wj, o.y, acc.y);
-        acc.z = fmaf(wj, o.z, acc.z);
-        acc.w = fmaf(wj, o.w, acc.w);
-      }
+    float mc = mj;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mc = fmaxf(mc, __shfl_xor_sync(0xFFFFFFFFu, mc, o));
+    const float M_new = fmaxf(M, mc);
+    if (M_new == -INFINITY) continue;
+    const float carry = (M == -INFINITY) ? 0.f : exp2f(M - M_new);
+    acc.x *= carry; acc.y *= carry; acc.z *= carry; acc.w *= carry;
+    L *= carry;
+    M = M_new;
+    const float w = (lj > 0.f) ? exp2f(mj - M) : 0.f;
+    const float wl = w * lj;
+    const int n = min(32, g.n_slots - j0);
+    for (int jb = 0; jb < n; jb += 8) {
+      float4 o[8];
+#pragma unroll
+      for (int k = 0; k < 8; ++k)
+        if (jb + k < n) o[k] = *reinterpret_cast<const float4 *>(tc.partial_o + (prow0 + (int64_t)(j0 + jb + k) * 128) * kD + lane * 4);
+#pragma unroll
+      for (int k = 0; k < 8; ++k)
+        if (jb + k < n) {
+          const float wj = __shfl_sync(0xFFFFFFFFu, w, jb + k);
+          L += __shfl_sync(0xFFFFFFFFu, wl, jb + k);
+          if (wj != 0.f) {
+            acc.x = fmaf(wj, o[k].x, acc.x);
+            acc.y = fmaf(wj, o[k].y, acc.y);
+            acc.z = fmaf(wj, o[k].z, acc.z);
+            acc.w = fmaf(wj, o[k].w, acc.w);
+          }
+        }
     }
   }
   const float inv = 1.0f / L;
@@ -646,9 +795,11 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t
                                   const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-int get_pool_map(lr_ctx *ctx, const void *pool, int64_t n_pages, const CUtensorMap **out) {
+// kind 0: a KV pool of n pages as [pages * kv heads * 16][128], box = one page half (16 rows x 64 channels)
+// kind 1: Q of n rows as [rows][q heads][128], box = 64 channels x G heads x T tokens
+int get_map(lr_ctx *ctx, int kind, const void *ptr, int64_t n, const CUtensorMap **out) {
   for (auto &e : ctx->tmaps)
-    if (e.ptr == pool && e.n_pages == n_pages) {
+    if (e.ptr == ptr && e.n == n && e.kind == kind) {
       *out = reinterpret_cast<const CUtensorMap *>(e.map);
       return LR_OK;
     }
@@ -665,17 +816,31 @@ int get_pool_map(lr_ctx *ctx, const void *pool, int64_t n_pages, const CUtensorM
   if (ctx->tmaps.size() >= 256) ctx->tmaps.erase(ctx->tmaps.begin());
   ctx->tmaps.emplace_back();
   lr_ctx::TmapEntry &ent = ctx->tmaps.back();
-  ent.ptr = pool;
-  ent.n_pages = n_pages;
-  // the pool as a 2-D tensor [rows = pages * kv heads * 16][128 channels]; a box is one page half: 16 rows x 64 channels
-  cuuint64_t dims[2] = {(cuuint64_t)kD, (cuuint64_t)n_pages * ctx->model.n_kv_heads * kPage};
-  cuuint64_t strides[1] = {(cuuint64_t)kD * 2};
-  cuuint32_t box[2] = {64, kPage};
-  cuuint32_t estr[2] = {1, 1};
-  CUresult r = reinterpret_cast<EncodeTiledFn>(ctx->tmap_encode)(
-      reinterpret_cast<CUtensorMap *>(ent.map), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(pool), dims, strides, box, estr,
-      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  ent.ptr = ptr;
+  ent.n = n;
+  ent.kind = kind;
+  const lr_model &m = ctx->model;
+  CUresult r;
+  if (kind == 0) {
+    cuuint64_t dims[2] = {(cuuint64_t)kD, (cuuint64_t)n * m.n_kv_heads * kPage};
+    cuuint64_t strides[1] = {(cuuint64_t)kD * 2};
+    cuuint32_t box[2] = {64, kPage};
+    cuuint32_t estr[2] = {1, 1};
+    r = reinterpret_cast<EncodeTiledFn>(ctx->tmap_encode)(
+        reinterpret_cast<CUtensorMap *>(ent.map), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(ptr), dims, strides, box,
+        estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  } else {
+    const int G = m.n_q_heads / m.n_kv_heads, T = 128 / G;
+    cuuint64_t dims[3] = {(cuuint64_t)kD, (cuuint64_t)m.n_q_heads, (cuuint64_t)n};
+    cuuint64_t strides[2] = {(cuuint64_t)kD * 2, (cuuint64_t)m.n_q_heads * kD * 2};
+    cuuint32_t box[3] = {64, (cuuint32_t)G, (cuuint32_t)T};
+    cuuint32_t estr[3] = {1, 1, 1};
+    r = reinterpret_cast<EncodeTiledFn>(ctx->tmap_encode)(
+        reinterpret_cast<CUtensorMap *>(ent.map), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(ptr), dims, strides, box,
+        estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  }
   if (r != CUDA_SUCCESS) {
     ctx->tmaps.pop_back();
     set_error("cuTensorMapEncodeTiled failed with CUresult %d", (int)r);
@@ -698,10 +863,13 @@ int tc_build_host_plan(const lr_ctx *ctx, const lr_batch *b, const int32_t *req_
   const lr_model &m = ctx->model;
   const int G = m.n_q_heads / m.n_kv_heads;
   if (m.head_dim != kD) return LR_OK;  // other head sizes take the CUDA-core path
+  if ((int64_t)b->n_pool_pages * m.n_kv_heads * kPage >= ((int64_t)1 << 31)) return LR_OK;  // tensor-map coordinates are 32-bit
   const int T = 128 / G;
+  const int n_q_rows = b->cu_q[b->n_branch];
   std::vector<TcPage> pages;
+  std::vector<TcRow> rows((size_t)std::max(1, n_q_rows));
   std::vector<TcReq> reqs((size_t)b->n_req);
-  struct Grp { int req, kv, mg, n_tiles, weight; };
+  struct Grp { int req, kv, mtile0, n_mt, n_tiles, weight, first_piece, n_pieces; };
   std::vector<Grp> grps;
   for (int r = 0; r < b->n_req; ++r) {
     const int s0 = b->req_span_off[r], s1 = b->req_span_off[r + 1];
@@ -709,14 +877,21 @@ int tc_build_host_plan(const lr_ctx *ctx, const lr_batch *b, const int32_t *req_
     TcReq &rq = reqs[r];
     memset(&rq, 0, sizeof(rq));
     rq.page_off = (int)pages.size();
-    rq.br0 = br0;
-    rq.n_br = br1 - br0;
-    if (rq.n_br == 0) continue;  // a request without branches has no query rows
-    if (rq.n_br > 254) return LR_OK;
+    if (br1 == br0) continue;  // a request without branches has no query rows
+    if (br1 - br0 > 254) return LR_OK;
     rq.q_row0 = b->cu_q[br0];
     rq.n_q = b->cu_q[br1] - b->cu_q[br0];
     int max_depth = 0;
-    for (int i = br0; i < br1; ++i) max_depth = std::max(max_depth, b->br_depth[i]);
+    for (int i = br0; i < br1; ++i) {
+      max_depth = std::max(max_depth, b->br_depth[i]);
+      if ((b->br_own_len[i] + kPage - 1) / kPage > 2047) return LR_OK;
+      const int q_len = b->cu_q[i + 1] - b->cu_q[i];
+      for (int k = 0; k < q_len; ++k) {
+        TcRow &w = rows[(size_t)b->cu_q[i] + k];
+        w.depth_branch = b->br_depth[i] | ((i - br0) << 16);
+        w.limit = b->br_own_len[i] - q_len + k;
+      }
+    }
     auto add_span = [&](int slot, int len, int need, int owner) {
       const int n = (len + kPage - 1) / kPage;
       for (int p = 0; p < n; ++p) {
@@ -726,10 +901,7 @@ int tc_build_host_plan(const lr_ctx *ctx, const lr_batch *b, const int32_t *req_
         e.meta = valid | ((uint32_t)need << 5) | ((uint32_t)owner << 13) | ((uint32_t)(owner ? p : 0) << 21);
         pages.push_back(e);
       }
-      return n;
     };
-    for (int i = br0; i < br1; ++i)
-      if ((b->br_own_len[i] + kPage - 1) / kPage > 2047) return LR_OK;
     add_span(b->span_slot[s0], b->span_len[s0], 0, 0);
     rq.n_dense_tiles = (b->span_len[s0] / kPage) / kPagesPerTile;
     for (int c = 1; c <= max_depth && s0 + c < s1; ++c) add_span(b->span_slot[s0 + c], b->span_len[s0 + c], c, 0);
@@ -737,11 +909,11 @@ int tc_build_host_plan(const lr_ctx *ctx, const lr_batch *b, const int32_t *req_
     rq.n_pages = (int)pages.size() - rq.page_off;
     while (pages.size() % kPagesPerTile) pages.push_back(TcPage{0, 0});  // absent pages of the last tile: nothing valid
     const int n_tiles = (rq.n_pages + kPagesPerTile - 1) / kPagesPerTile;
-    const int n_mt = (rq.n_q + T - 1) / T;
+    const int n_mtiles = (rq.n_q + T - 1) / T;
     for (int kv = 0; kv < m.n_kv_heads; ++kv)
-      for (int mg = 0; mg < (n_mt + 1) / 2; ++mg) {
-        const int mts = std::min(2, n_mt - 2 * mg);
-        grps.push_back(Grp{r, kv, mg, n_tiles, 1 + mts});
+      for (int m0 = 0; m0 < n_mtiles; m0 += 2) {
+        const int mts = std::min(2, n_mtiles - m0);
+        grps.push_back(Grp{r, kv, m0, mts, n_tiles, 1 + mts, 0, 0});
       }
   }
   if (grps.empty()) return LR_OK;
@@ -755,61 +927,70 @@ int tc_build_host_plan(const lr_ctx *ctx, const lr_batch *b, const int32_t *req_
   const int n_cta = (int)std::min<int64_t>(ctx->sm_count, std::max<int64_t>(1, total_tiles / 2));
   std::vector<TcPiece> pieces;
   std::vector<int32_t> cta_off((size_t)n_cta + 1, 0);
-  std::vector<TcGroup> groups(grps.size());
+  std::vector<int> piece_group;
   int64_t w_pos = 0;
   int cta = 0, last_cta = -1;
   for (size_t gi = 0; gi < grps.size(); ++gi) {
-    const Grp &g = grps[gi];
-    const int first_piece = (int)pieces.size();
+    Grp &g = grps[gi];
+    g.first_piece = (int)pieces.size();
     for (int t = 0; t < g.n_tiles; ++t, w_pos += g.weight) {
       while (cta + 1 < n_cta && w_pos >= total_w * (cta + 1) / n_cta) {
         ++cta;
         cta_off[cta] = (int32_t)pieces.size();
       }
-      if (!pieces.empty() && pieces.back().group_id == (int)gi && last_cta == cta) {
+      if (!pieces.empty() && piece_group.back() == (int)gi && last_cta == cta) {
         pieces.back().tile_end = t + 1;  // same group, same CTA: extend the piece
       } else {
         TcPiece p;
-        p.req = g.req; p.kv_head = g.kv; p.mgroup = g.mg; p.tile_begin = t; p.tile_end = t + 1;
-        p.partial_slot = -1; p.group_id = (int)gi; p.pad = 0;
+        p.req = g.req; p.kv_head = g.kv; p.mtile0 = g.mtile0; p.n_mt = g.n_mt; p.tile_begin = t; p.tile_end = t + 1;
+        p.slot[0] = p.slot[1] = -2;
         pieces.push_back(p);
+        piece_group.push_back((int)gi);
         last_cta = cta;
       }
     }
-    TcGroup &tg = groups[gi];
-    memset(&tg, 0, sizeof(tg));
-    tg.req = g.req; tg.kv_head = g.kv; tg.mgroup = g.mg;
-    tg.n_partial = (int)pieces.size() - first_piece;
-    tg.partial_begin = first_piece;  // provisional: index of the group's first piece
+    g.n_pieces = (int)pieces.size() - g.first_piece;
   }
   for (int c = cta + 1; c <= n_cta; ++c) cta_off[c] = (int32_t)pieces.size();
-  // partial slots for groups cut into several pieces
+  // Targets (one M-tile of one group) and the streams that contribute to them, in piece order.
   int n_slots = 0;
-  std::vector<TcGroup> merge_groups;
-  for (size_t gi = 0; gi < grps.size(); ++gi) {
-    TcGroup &tg = groups[gi];
-    if (tg.n_partial >= 2) {
-      const int first_piece = tg.partial_begin;
-      tg.partial_begin = n_slots;
-      for (int k = 0; k < tg.n_partial; ++k) pieces[first_piece + k].partial_slot = n_slots++;
-      merge_groups.push_back(tg);
+  std::vector<TcTarget> targets;
+  for (const Grp &g : grps)
+    for (int mt = 0; mt < g.n_mt; ++mt) {
+      std::vector<int32_t *> contrib;
+      for (int k = 0; k < g.n_pieces; ++k) {
+        TcPiece &p = pieces[g.first_piece + k];
+        const int n = p.tile_end - p.tile_begin;
+        if (g.n_mt == 2) contrib.push_back(&p.slot[mt]);
+        else {
+          contrib.push_back(&p.slot[0]);
+          if (n >= 2) contrib.push_back(&p.slot[1]);
+        }
+      }
+      if (contrib.size() == 1) { *contrib[0] = -1; continue; }
+      TcTarget tg;
+      memset(&tg, 0, sizeof(tg));
+      tg.req = g.req; tg.kv_head = g.kv; tg.mtile = g.mtile0 + mt;
+      tg.slot_begin = n_slots; tg.n_slots = (int)contrib.size();
+      for (int32_t *c : contrib) *c = n_slots++;
+      targets.push_back(tg);
     }
-  }
   out.ok = true;
   out.n_cta = n_cta;
   out.n_pieces = (int)pieces.size();
-  out.n_groups = n_slots ? (int)merge_groups.size() : 0;
+  out.n_targets = (int)targets.size();
   out.n_partial_slots = n_slots;
   out.tokens_per_mtile = T;
   out.o_pages = img.add(pages.data(), pages.size() * sizeof(TcPage));
+  out.o_rows = img.add(rows.data(), rows.size() * sizeof(TcRow));
   out.o_pieces = img.add(pieces.data(), pieces.size() * sizeof(TcPiece));
   out.o_cta_piece_off = img.add(cta_off.data(), cta_off.size() * sizeof(int32_t));
   out.o_reqs = img.add(reqs.data(), reqs.size() * sizeof(TcReq));
-  if (merge_groups.empty()) merge_groups.push_back(TcGroup{});  // keep the section non-empty
-  out.o_groups = img.add(merge_groups.data(), merge_groups.size() * sizeof(TcGroup));
+  if (targets.empty()) targets.push_back(TcTarget{});  // keep the section non-empty
+  out.o_targets = img.add(targets.data(), targets.size() * sizeof(TcTarget));
   out.s_ml = 0;
-  out.s_o = ((size_t)n_slots * 256 * 2 * sizeof(float) + 255) / 256 * 256;
-  out.scratch_bytes = out.s_o + (size_t)n_slots * 256 * kD * sizeof(float);
+  out.s_o = ((size_t)n_slots * 128 * 2 * sizeof(float) + 255) / 256 * 256;
+  out.scratch_bytes = out.s_o + (size_t)n_slots * 128 * kD * sizeof(float);
   out.scratch_zero_bytes = 0;
   return LR_OK;
 }
@@ -820,36 +1001,48 @@ void tc_bind_device_plan(const TcHostPlan &h, unsigned char *image_base, unsigne
   if (!h.ok) return;
   DevTcPlan &t = p->tc;
   t.pages = reinterpret_cast<const TcPage *>(image_base + h.o_pages);
+  t.rows = reinterpret_cast<const TcRow *>(image_base + h.o_rows);
   t.pieces = reinterpret_cast<const TcPiece *>(image_base + h.o_pieces);
   t.cta_piece_off = reinterpret_cast<const int32_t *>(image_base + h.o_cta_piece_off);
   t.reqs = reinterpret_cast<const TcReq *>(image_base + h.o_reqs);
-  t.groups = reinterpret_cast<const TcGroup *>(image_base + h.o_groups);
+  t.targets = reinterpret_cast<const TcTarget *>(image_base + h.o_targets);
   t.n_cta = h.n_cta;
-  t.n_groups = h.n_groups;
-  t.n_merge_groups = h.n_groups;
+  t.n_targets = h.n_targets;
   t.tokens_per_mtile = h.tokens_per_mtile;
   t.partial_ml = reinterpret_cast<float *>(scratch_base + h.s_ml);
   t.partial_o = reinterpret_cast<float *>(scratch_base + h.s_o);
-  t.tickets = nullptr;
 }
 
 int launch_attn_tc(lr_plan *p, const void *q, const void *k, const void *v, void *out, float *lse, float scale,
                    cudaStream_t s) {
-  const CUtensorMap *km = nullptr, *vm = nullptr;
-  if (int rc = get_pool_map(p->ctx, k, p->dev.n_pool_pages, &km)) return rc;
-  CUtensorMap kmap = *km;  // the cache may reallocate when the second map is added
-  if (int rc = get_pool_map(p->ctx, v, p->dev.n_pool_pages, &vm)) return rc;
-  CUtensorMap vmap = *vm;
+  const CUtensorMap *mp = nullptr;
+  if (int rc = get_map(p->ctx, 0, k, p->dev.n_pool_pages, &mp)) return rc;
+  const CUtensorMap kmap = *mp;  // the cache may reallocate when the next map is added
+  if (int rc = get_map(p->ctx, 0, v, p->dev.n_pool_pages, &mp)) return rc;
+  const CUtensorMap vmap = *mp;
+  if (int rc = get_map(p->ctx, 1, q, p->dev.n_q_rows, &mp)) return rc;
+  const CUtensorMap qmap = *mp;
   const float scale_log2 = scale * 1.4426950408889634f;
-  attn_tc_kernel<<<p->tc.n_cta, kThreads, kSmemBytes, s>>>(kmap, vmap, p->dev, p->tc, reinterpret_cast<const uint16_t *>(q),
-                                                            reinterpret_cast<uint16_t *>(out), lse, scale_log2);
+  attn_tc_kernel<<<p->tc.n_cta, kThreads, kSmemBytes, s>>>(kmap, vmap, qmap, p->dev, p->tc, reinterpret_cast<uint16_t *>(out), lse,
+                                                            scale_log2);
   p->ctx->launches++;
   if (int rc = cuda_fail(cudaGetLastError(), "attn_tc_kernel launch")) return rc;
-  if (p->tc.n_merge_groups > 0) {
-    dim3 grid((unsigned)p->tc.n_merge_groups, 32);
-    attn_tc_merge_kernel<<<grid, 256, 0, s>>>(p->dev, p->tc, reinterpret_cast<uint16_t *>(out), lse);
+  if (p->tc.n_targets > 0) {
+    // programmatic dependent launch: the merge grid is set up while the attention grid drains
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3((unsigned)p->tc.n_targets, 16, 1);
+    cfg.blockDim = dim3(256, 1, 1);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, attn_tc_merge_kernel, p->dev, p->tc, reinterpret_cast<uint16_t *>(out), lse);
     p->ctx->launches++;
-    if (int rc = cuda_fail(cudaGetLastError(), "attn_tc_merge_kernel launch")) return rc;
+    if (int rc = cuda_fail(e, "attn_tc_merge_kernel launch")) return rc;
   }
   return LR_OK;
 }

@@ -37,43 +37,50 @@ struct DevBatch {
 // ---- tensor-core attention plan (device side) -------------------------------
 // A request's *extended chain* is the list of its page slots in the order
 // prefix, segments 1..gamma, branch tails; consecutive groups of 8 pages form
-// 128-key tiles.  An (request, kv head, M-group) triple is a *group*; its tiles
-// are cut into contiguous *pieces*, one or more per CTA.
+// 128-key tiles.  The query rows that share one KV head -- (query token, head in
+// group) pairs -- are packed into 128-row M-tiles.  A *group* is (request, KV
+// head, one or two M-tiles); its tiles are cut into contiguous *pieces*, one or
+// more per CTA.  A CTA runs two independent streams: the two M-tiles of the
+// piece, or -- for a piece with one M-tile -- its even and odd tiles.  A
+// *target* is one M-tile of one (request, KV head); when several streams
+// contribute to a target each writes an fp32 partial and a second kernel merges.
 struct TcPage {      // one per extended-chain page
   int32_t page;      // physical page id
-  uint32_t meta;     // bits 0-4 valid tokens (1..16), 5-12 min depth to see it, 13-20 owner branch (local, +1; 0 = chain), 21-31 first tail token index of the page / 16
+  uint32_t meta;     // bits 0-4 valid tokens (0..16), 5-12 min depth to see it, 13-20 owner branch (local, +1; 0 = chain), 21-31 first tail token index of the page / 16
+};
+struct TcRow {       // one per query row of the batch
+  int32_t depth_branch;  // depth | local branch index << 16
+  int32_t limit;         // last tail token the row sees
 };
 struct TcPiece {
-  int32_t req, kv_head, mgroup;   // which rows x which KV head
+  int32_t req, kv_head;
+  int32_t mtile0, n_mt;           // first M-tile and how many (1 or 2)
   int32_t tile_begin, tile_end;   // tiles of the request's extended chain
-  int32_t partial_slot;           // < 0: sole piece of its group, write final output directly
-  int32_t group_id;
-  int32_t pad;
+  int32_t slot[2];                // per stream: >= 0 partial slot, -1 write the final output, -2 nothing to write
 };
 struct TcReq {
   int32_t page_off;     // first TcPage of the request
   int32_t n_pages;      // extended-chain pages
   int32_t q_row0, n_q;  // query token range of the request
-  int32_t br0, n_br;    // branch range
   int32_t n_dense_tiles;  // leading tiles made only of full prefix pages (no masking needed)
-  int32_t pad;
+  int32_t pad[3];
 };
-struct TcGroup {
-  int32_t req, kv_head, mgroup;
-  int32_t partial_begin, n_partial;  // partial slots to merge (n_partial >= 2), else unused
+struct TcTarget {
+  int32_t req, kv_head, mtile;
+  int32_t slot_begin, n_slots;  // partial slots to merge (n_slots >= 2)
   int32_t pad[3];
 };
 struct DevTcPlan {
   const TcPage *pages;
+  const TcRow *rows;             // [n_q_rows]
   const TcPiece *pieces;
   const int32_t *cta_piece_off;  // [n_cta+1]
   const TcReq *reqs;
-  const TcGroup *groups;
-  int32_t n_cta, n_groups, n_merge_groups;
+  const TcTarget *targets;
+  int32_t n_cta, n_targets;
   int32_t tokens_per_mtile;  // floor(128 / group)
-  float *partial_o;          // [n_partial_slots][256][head_dim] fp32, unnormalised
-  float *partial_ml;         // [n_partial_slots][256][2] (running max in log2 units, sum)
-  int32_t *tickets;          // [n_groups], zero between launches
+  float *partial_o;          // [n_slots][128][head_dim] fp32, unnormalised
+  float *partial_ml;         // [n_slots][128][2] (reference exponent in log2 units, sum)
 };
 
 }  // namespace lr
@@ -84,7 +91,7 @@ struct lr_ctx {
   int sm_count;
   int64_t launches;
   void *tmap_encode;  // cuTensorMapEncodeTiled entry point (driver), resolved lazily
-  struct TmapEntry { const void *ptr; int64_t n_pages; alignas(64) unsigned char map[128]; };
+  struct TmapEntry { const void *ptr; int64_t n; int kind; alignas(64) unsigned char map[128]; };
   std::vector<TmapEntry> tmaps;
 };
 
@@ -120,10 +127,10 @@ struct Image {
 // Host-side result of planning the tensor-core attention for one batch.
 struct TcHostPlan {
   bool ok = false;  // shape supported by the tensor-core path
-  size_t o_pages = 0, o_pieces = 0, o_cta_piece_off = 0, o_reqs = 0, o_groups = 0;  // image offsets
-  int n_cta = 0, n_groups = 0, n_pieces = 0, n_partial_slots = 0, tokens_per_mtile = 0;
-  // scratch region behind the image: tickets (zeroed at plan creation), then (max, sum) pairs, then fp32 partial outputs
-  size_t s_tickets = 0, s_ml = 0, s_o = 0, scratch_bytes = 0, scratch_zero_bytes = 0;
+  size_t o_pages = 0, o_rows = 0, o_pieces = 0, o_cta_piece_off = 0, o_reqs = 0, o_targets = 0;  // image offsets
+  int n_cta = 0, n_targets = 0, n_pieces = 0, n_partial_slots = 0, tokens_per_mtile = 0;
+  // scratch region behind the image: (exponent, sum) pairs, then fp32 partial outputs
+  size_t s_ml = 0, s_o = 0, scratch_bytes = 0, scratch_zero_bytes = 0;
 };
 int tc_build_host_plan(const lr_ctx *ctx, const lr_batch *b, const int32_t *req_br_off, TcHostPlan &out, Image &img);
 void tc_bind_device_plan(const TcHostPlan &h, unsigned char *image_base, unsigned char *scratch_base, lr_plan *p);
