@@ -1,14 +1,19 @@
 // Greedy token-level acceptance: one streaming pass over the bf16 logits.
 //
-// Grid (chunks of a row, rows).  Each CTA reduces 8192 consecutive logits of
-// one row to (max value, lowest index), publishes it with one 64-bit atomicMax
-// on the row's key and takes a ticket; the CTA holding the last ticket turns the
-// row keys into n_accept / bonus per branch and zeroes the scratch again.
+// The logits are cut into equal contiguous ranges of 16-byte vectors, one per CTA
+// of a fixed grid (a few CTAs per SM), whatever the row boundaries; a range that
+// spans several rows is handled row segment by row segment.  Each segment is
+// reduced to (max value, lowest index) and published with one 64-bit atomicMax
+// on the row's key; a CTA then takes a ticket, and the one holding the last
+// ticket turns the row keys into n_accept / bonus per branch and zeroes the
+// scratch again.
 //
 // The work is bound by HBM reads: 2 bytes per logit, read once, 16-byte loads,
-// four independent loads in flight per thread.  The maximum is taken with
+// eight independent loads in flight per thread.  The maximum is taken with
 // packed bf16x2 max instructions on whole 16-byte vectors (about one
 // instruction per logit); the index is resolved only inside the winning vector.
+#include <algorithm>
+
 #include "lr_common.cuh"
 
 namespace lr {
@@ -16,8 +21,8 @@ namespace lr {
 namespace {
 
 constexpr int kThreads = 256;
-constexpr int kVecPerThread = 4;                          // 16-byte vectors per thread per CTA
-constexpr int kChunk = kThreads * kVecPerThread * 8;      // logits per CTA
+constexpr int kVecPerThread = 8;                          // 16-byte vectors in flight per thread
+constexpr int kCtasPerSm = 4;
 
 // Monotone map of a float (already NaN-free, -0 folded to +0) to an unsigned key.
 __device__ __forceinline__ uint32_t order_key(float x) {
@@ -85,81 +90,97 @@ accept_greedy_kernel(const uint16_t *__restrict__ logits, int64_t row_stride, in
                      int32_t *__restrict__ row_argmax, unsigned long long *scratch) {
   unsigned int *counter = reinterpret_cast<unsigned int *>(scratch);
   unsigned long long *row_key = scratch + 1;
-  const int row = blockIdx.y;
   const int tid = threadIdx.x;
-  const int64_t c0 = (int64_t)blockIdx.x * kChunk;
-  const uint16_t *rp = logits + (int64_t)row * row_stride;
-  const int32_t n_vec = vocab >> 3;  // whole 16-byte vectors in the row
+  const int32_t n_vec = vocab >> 3;  // whole 16-byte vectors in a row
+  // A row is n_vec vector units plus one unit for its ragged end (vocab not a multiple of 8).
+  const int64_t upr = (int64_t)n_vec + 1, total = upr * n_rows;
+  const int64_t per = (total + gridDim.x - 1) / gridDim.x;
+  int64_t pos = (int64_t)blockIdx.x * per;
+  const int64_t end = min(total, pos + per);
+  __shared__ float s_v[kThreads / 32];
+  __shared__ int32_t s_i[kThreads / 32];
+  __shared__ int s_last;
+  asm volatile("griddepcontrol.wait;" ::: "memory");  // the logits may come from the kernel launched just before
 
-  // Per thread: vectors are visited in increasing index order and only a strictly
-  // greater maximum replaces the current one, so the earliest maximum is kept.
-  Best best;
-  best.v = -INFINITY;
-  best.i = 0x7FFFFFFF;  // "owns no element": loses every tie
-  {
+  while (pos < end) {
+    const int row = (int)(pos / upr);
+    const int32_t u0 = (int32_t)(pos - (int64_t)row * upr);
+    const int32_t u1 = (int32_t)min(upr, (int64_t)u0 + (end - pos));
+    const int32_t v_end = min(u1, n_vec);
+    const uint16_t *rp = logits + (int64_t)row * row_stride;
     const uint4 *vp = reinterpret_cast<const uint4 *>(rp);
-    uint4 v[kVecPerThread];
-    int32_t vi[kVecPerThread];
-#pragma unroll
-    for (int k = 0; k < kVecPerThread; ++k) {
-      vi[k] = (int32_t)(c0 >> 3) + k * kThreads + tid;
-      if (vi[k] < n_vec) v[k] = ld_stream(vp + vi[k]);
-    }
+    // Per thread: vectors are visited in increasing index order and only a strictly
+    // greater maximum replaces the current one, so the earliest maximum is kept.
+    Best best;
+    best.v = -INFINITY;
+    best.i = 0x7FFFFFFF;  // "owns no element": loses every tie
     uint4 bv = make_uint4(0, 0, 0, 0);
     int32_t bvi = -1;
+    for (int32_t base = u0; base < v_end; base += kThreads * kVecPerThread) {
+      uint4 v[kVecPerThread];
 #pragma unroll
-    for (int k = 0; k < kVecPerThread; ++k) {
-      if (vi[k] < n_vec) {
-        float m = denan(vec_max(v[k]));
-        if (m > best.v || bvi < 0) {
-          best.v = m;
-          bv = v[k];
-          bvi = vi[k];
+      for (int k = 0; k < kVecPerThread; ++k) {
+        const int32_t vi = base + k * kThreads + tid;
+        if (vi < v_end) v[k] = ld_stream(vp + vi);
+      }
+#pragma unroll
+      for (int k = 0; k < kVecPerThread; ++k) {
+        const int32_t vi = base + k * kThreads + tid;
+        if (vi < v_end) {
+          const float m = denan(vec_max(v[k]));
+          if (m > best.v || bvi < 0) {
+            best.v = m;
+            bv = v[k];
+            bvi = vi;
+          }
         }
       }
     }
     // a maximum of -inf means every element is -inf or NaN: the first one wins
     if (bvi >= 0) best.i = bvi * 8 + (best.v == -INFINITY ? 0 : first_equal(bv, best.v));
-  }
-  // ragged end of the row (vocab not a multiple of 8): up to 7 single elements
-  if (blockIdx.x == gridDim.x - 1) {
-    int32_t e = n_vec * 8 + tid;
-    if (e < vocab) {
-      Best t;
-      t.v = denan(bf_lo((uint32_t)rp[e]));
-      t.i = e;
-      best = better(best, t);
+    // ragged end of the row: up to 7 single elements
+    if (u1 == (int32_t)upr) {
+      const int32_t e = n_vec * 8 + tid;
+      if (e < vocab) {
+        Best t;
+        t.v = denan(bf_lo((uint32_t)rp[e]));
+        t.i = e;
+        best = better(best, t);
+      }
     }
-  }
-  // warp, then block reduction
+    // warp, then block reduction
 #pragma unroll
-  for (int off = 16; off > 0; off >>= 1) {
-    Best o;
-    o.v = __shfl_down_sync(0xFFFFFFFFu, best.v, off);
-    o.i = __shfl_down_sync(0xFFFFFFFFu, best.i, off);
-    best = better(best, o);
-  }
-  __shared__ float s_v[kThreads / 32];
-  __shared__ int32_t s_i[kThreads / 32];
-  __shared__ int s_last;
-  if ((tid & 31) == 0) {
-    s_v[tid >> 5] = best.v;
-    s_i[tid >> 5] = best.i;
-  }
-  __syncthreads();
-  if (tid == 0) {
-    for (int w = 1; w < kThreads / 32; ++w) {
+    for (int off = 16; off > 0; off >>= 1) {
       Best o;
-      o.v = s_v[w];
-      o.i = s_i[w];
+      o.v = __shfl_down_sync(0xFFFFFFFFu, best.v, off);
+      o.i = __shfl_down_sync(0xFFFFFFFFu, best.i, off);
       best = better(best, o);
     }
-    unsigned long long key = ((unsigned long long)order_key(best.v) << 32) | (unsigned long long)(0xFFFFFFFFu - (uint32_t)best.i);
-    atomicMax(row_key + row, key);
+    if ((tid & 31) == 0) {
+      s_v[tid >> 5] = best.v;
+      s_i[tid >> 5] = best.i;
+    }
+    __syncthreads();
+    if (tid == 0) {
+      for (int w = 1; w < kThreads / 32; ++w) {
+        Best o;
+        o.v = s_v[w];
+        o.i = s_i[w];
+        best = better(best, o);
+      }
+      if (best.i != 0x7FFFFFFF) {
+        unsigned long long key =
+            ((unsigned long long)order_key(best.v) << 32) | (unsigned long long)(0xFFFFFFFFu - (uint32_t)best.i);
+        atomicMax(row_key + row, key);
+      }
+    }
+    __syncthreads();
+    pos += u1 - u0;
+  }
+  if (tid == 0) {
     __threadfence();
-    unsigned int total = gridDim.x * gridDim.y;
     unsigned int t = atomicAdd(counter, 1u);
-    s_last = (t == total - 1);
+    s_last = (t == gridDim.x - 1);
   }
   __syncthreads();
   if (!s_last) return;
@@ -225,15 +246,13 @@ int launch_accept(lr_ctx *ctx, const void *logits, int64_t stride, const int32_t
                   int32_t n_branch, int32_t n_rows, int32_t *n_accept, int32_t *bonus, int32_t *row_argmax,
                   void *scratch, cudaStream_t s) {
   const int32_t vocab = ctx->model.vocab;
-  const unsigned chunks = (unsigned)((vocab + kChunk - 1) / kChunk);
-  if (n_rows > 65535) {
-    set_error("lr_accept_greedy: more than 65535 logits rows in one call");
-    return LR_EUNSUPPORTED;
-  }
-  dim3 grid(chunks, (unsigned)n_rows);
-  accept_greedy_kernel<<<grid, kThreads, 0, s>>>(reinterpret_cast<const uint16_t *>(logits), stride, vocab, drafts,
-                                                  cu_draft, n_branch, n_rows, n_accept, bonus, row_argmax,
-                                                  reinterpret_cast<unsigned long long *>(scratch));
+  // equal ranges of at least one full round of loads per CTA, at most kCtasPerSm CTAs per SM
+  const int64_t total = ((int64_t)(vocab >> 3) + 1) * n_rows;
+  int64_t grid = (total + kThreads * kVecPerThread - 1) / (kThreads * kVecPerThread);
+  grid = std::max<int64_t>(1, std::min<int64_t>(grid, (int64_t)ctx->sm_count * kCtasPerSm));
+  accept_greedy_kernel<<<(unsigned)grid, kThreads, 0, s>>>(reinterpret_cast<const uint16_t *>(logits), stride, vocab, drafts,
+                                                            cu_draft, n_branch, n_rows, n_accept, bonus, row_argmax,
+                                                            reinterpret_cast<unsigned long long *>(scratch));
   ctx->launches++;
   return cuda_fail(cudaGetLastError(), "accept_greedy_kernel launch");
 }

@@ -1,10 +1,14 @@
 // Step-level commit on the paged KV cache (Algorithm 1, last two lines).
 //
 // Integer work on a few KB of tables: latency-bound, so it is one launch with no
-// inter-CTA communication.  Every CTA recomputes the per-request decisions
-// (j*, decisive branch, kept tail, list sizes) and their exclusive scans in
-// shared memory -- O(requests x gamma) work -- and then the warps of all CTAs
-// share the page-list writes, one warp per span or branch tail.
+// inter-CTA communication and as few dependent loads as possible.  Every CTA
+// recomputes the per-request decisions (j*, decisive branch, kept tail, list
+// sizes) -- one thread per request, with the verdict and depth scans unrolled in
+// groups of 8 so that their loads are in flight together -- and the exclusive
+// scans of the list sizes in shared memory.  The page lists are then written
+// one thread per page slot: the plan holds, for every slot, the span or tail
+// that owns it and prefix sums of pages per request, so a slot's place in the
+// keep or free list is a handful of independent loads and adds.
 #include "lr_common.cuh"
 
 namespace lr {
@@ -13,10 +17,11 @@ namespace {
 
 constexpr int kThreads = 256;
 constexpr int kMaxReq = 4096;
+constexpr int kSmemPerReq = 7 * 4;  // bytes of shared memory per request
 
 __device__ __forceinline__ int pages_of(int n_tok) { return (n_tok + kPage - 1) / kPage; }
 
-// exclusive scan of a[0..n) in shared memory, in place, by one CTA; returns nothing, total in *total
+// exclusive scan of a[0..n) in shared memory, in place, by one CTA; the total goes to *carry_slot
 __device__ void block_exclusive_scan(int32_t *a, int n, int32_t *carry_slot) {
   __shared__ int32_t warp_sum[kThreads / 32];
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
@@ -54,41 +59,59 @@ commit_kernel(DevBatch d, const uint8_t *__restrict__ verdict,
   int32_t *s_free = sm + R;        // free count -> free offset
   int32_t *s_a = sm + 2 * R;       // j*
   int32_t *s_surv = sm + 3 * R;    // decisive branch or -1
+  int32_t *s_kp = sm + 4 * R;      // kept tail pages of the decisive branch
+  int32_t *s_kt = sm + 5 * R;      // kept tail tokens
+  int32_t *s_kchain = sm + 6 * R;  // pages of the kept chain spans (prefix and segments 1..j*)
   __shared__ int32_t s_total[2];
   const int tid = threadIdx.x;
+  asm volatile("griddepcontrol.wait;" ::: "memory");  // n_accept comes from the kernel launched just before
 
   // ---- per-request decisions --------------------------------------------------
   for (int r = tid; r < R; r += kThreads) {
     const int s0 = d.req_span_off[r], s1 = d.req_span_off[r + 1];
-    const int gamma = s1 - s0 - 1;
+    const int b0 = d.req_br_off[r], b1 = d.req_br_off[r + 1];
+    const int gamma = s1 - s0 - 1, base = s0 + r;
     const uint8_t *v = verdict + (s0 - r);
-    int a = 0;
-    while (a < gamma && v[a] != 0) ++a;  // j* = first rejected step, gamma if none
-    int surv = -1;
-    for (int b = d.req_br_off[r]; b < d.req_br_off[r + 1]; ++b)
-      if (d.br_depth[b] == a) { surv = b; break; }
+    int a = gamma;  // j* = first rejected step, gamma if none
+    for (int c0 = 0; c0 < gamma && a == gamma; c0 += 8) {
+      uint8_t w[8];
+#pragma unroll
+      for (int k = 0; k < 8; ++k) w[k] = (c0 + k < gamma) ? v[c0 + k] : (uint8_t)1;
+#pragma unroll
+      for (int k = 7; k >= 0; --k)
+        if (w[k] == 0) a = c0 + k;
+    }
+    int surv = -1;  // lowest-numbered branch of depth j*
+    for (int i0 = b0; i0 < b1 && surv < 0; i0 += 8) {
+      int dep[8];
+#pragma unroll
+      for (int k = 0; k < 8; ++k) dep[k] = (i0 + k < b1) ? d.br_depth[i0 + k] : -1;
+#pragma unroll
+      for (int k = 7; k >= 0; --k)
+        if (dep[k] == a) surv = i0 + k;
+    }
     int kept_tail = 0;
     if (surv >= 0) {
-      int L = d.br_n_draft[surv];
+      const int L = d.br_n_draft[surv], own = d.br_own_len[surv];
       int na = n_accept[surv];
       if (na < 0 || na > L) {  // not a value the acceptance step can produce
         na = na < 0 ? 0 : L;
         d.status[0] = kDevBounds;
-        d.status[1] = 300 + 0;
+        d.status[1] = 300;
       }
-      kept_tail = d.br_own_len[surv] - L + na;
+      kept_tail = own - L + na;
     }
-    int keep = pages_of(kept_tail), total = 0, len = kept_tail;
-    for (int c = 0; c <= gamma; ++c) {
-      int pg = pages_of(d.span_len[s0 + c]);
-      total += pg;
-      if (c <= a) { keep += pg; len += d.span_len[s0 + c]; }
-    }
-    for (int b = d.req_br_off[r]; b < d.req_br_off[r + 1]; ++b) total += pages_of(d.br_own_len[b]);
-    s_keep[r] = keep;
-    s_free[r] = total - keep;
+    const int kchain = d.chain_pg[base + a + 1], chain_all = d.chain_pg[base + gamma + 1];
+    const int tails_all = d.tail_pg[b0 + r + (b1 - b0)];
+    const int len = d.chain_tok[base + a + 1] + kept_tail;
+    const int kp = pages_of(kept_tail);
+    s_keep[r] = kchain + kp;
+    s_free[r] = chain_all + tails_all - kchain - kp;
     s_a[r] = a;
     s_surv[r] = surv;
+    s_kp[r] = kp;
+    s_kt[r] = kept_tail;
+    s_kchain[r] = kchain;
     if (blockIdx.x == 0) {
       n_steps_out[r] = a;
       survivor_out[r] = surv;
@@ -109,52 +132,37 @@ commit_kernel(DevBatch d, const uint8_t *__restrict__ verdict,
     }
   }
 
-  // ---- page lists: one warp per span / branch tail ---------------------------------
-  const int lane = tid & 31;
-  const int warps_total = gridDim.x * (kThreads / 32);
-  const int n_items = d.n_span + d.n_branch;
-  for (int item = blockIdx.x * (kThreads / 32) + (tid >> 5); item < n_items; item += warps_total) {
+  // ---- page lists: one thread per page slot --------------------------------------
+  for (int i = blockIdx.x * kThreads + tid; i < d.n_page_slots; i += gridDim.x * kThreads) {
+    const int item = d.slot_item[i];
+    if (item < 0) continue;  // a slot no span refers to
+    const int32_t pid = d.page_ids[i];
     if (item < d.n_span) {
       const int s = item, r = d.span_req[s];
       const int s0 = d.req_span_off[r], c = s - s0, a = s_a[r];
-      const int len = d.span_len[s], npg = pages_of(len);
-      const int32_t *src = d.page_ids + d.span_slot[s];
+      const int idx = i - d.span_slot[s], before = d.chain_pg[s0 + r + c];
       if (c <= a) {
-        int off = s_keep[r];
-        for (int cc = 0; cc < c; ++cc) off += pages_of(d.span_len[s0 + cc]);
-        for (int p = lane; p < npg; p += 32) {
-          keep_pages[off + p] = src[p];
-          keep_valid[off + p] = min(kPage, len - p * kPage);
-        }
+        const int dst = s_keep[r] + before + idx;
+        keep_pages[dst] = pid;
+        keep_valid[dst] = min(kPage, d.span_len[s] - idx * kPage);
       } else {
-        int off = s_free[r];
-        for (int cc = a + 1; cc < c; ++cc) off += pages_of(d.span_len[s0 + cc]);
-        for (int p = lane; p < npg; p += 32) free_pages[off + p] = src[p];
+        free_pages[s_free[r] + before - s_kchain[r] + idx] = pid;
       }
     } else {
       const int b = item - d.n_span, r = d.br_req[b];
-      const int s0 = d.req_span_off[r], s1 = d.req_span_off[r + 1], a = s_a[r], surv = s_surv[r];
-      int kept_tail = 0, kp = 0;
-      if (surv >= 0) {
-        int L = d.br_n_draft[surv], na = min(max(n_accept[surv], 0), L);
-        kept_tail = d.br_own_len[surv] - L + na;
-        kp = pages_of(kept_tail);
+      const int s0 = d.req_span_off[r], s1 = d.req_span_off[r + 1], b0 = d.req_br_off[r];
+      const int surv = s_surv[r], kp = s_kp[r], kchain = s_kchain[r];
+      const int idx = i - d.br_own_slot[b];
+      if (b == surv && idx < kp) {
+        const int dst = s_keep[r] + kchain + idx;
+        keep_pages[dst] = pid;
+        keep_valid[dst] = min(kPage, s_kt[r] - idx * kPage);
+      } else {
+        const int chain_free = d.chain_pg[s0 + r + (s1 - s0)] - kchain;
+        const int tails_before = d.tail_pg[b0 + r + (b - b0)];
+        const int kept_before = (surv >= 0 && b >= surv) ? kp : 0;  // kept pages precede this one in tail order
+        free_pages[s_free[r] + chain_free + tails_before - kept_before + idx] = pid;
       }
-      const int npg = pages_of(d.br_own_len[b]);
-      const int32_t *src = d.page_ids + d.br_own_slot[b];
-      if (b == surv) {
-        int off = s_keep[r];
-        for (int c = 0; c <= a; ++c) off += pages_of(d.span_len[s0 + c]);
-        for (int p = lane; p < kp; p += 32) {
-          keep_pages[off + p] = src[p];
-          keep_valid[off + p] = min(kPage, kept_tail - p * kPage);
-        }
-      }
-      int off = s_free[r];
-      for (int c = a + 1; c < s1 - s0; ++c) off += pages_of(d.span_len[s0 + c]);
-      for (int bb = d.req_br_off[r]; bb < b; ++bb) off += pages_of(d.br_own_len[bb]) - (bb == surv ? kp : 0);
-      const int skip = (b == surv) ? kp : 0;
-      for (int p = skip + lane; p < npg; p += 32) free_pages[off + p - skip] = src[p];
     }
   }
 }
@@ -162,7 +170,7 @@ commit_kernel(DevBatch d, const uint8_t *__restrict__ verdict,
 }  // namespace
 
 int init_commit_kernel() {
-  return cuda_fail(cudaFuncSetAttribute(commit_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxReq * 16),
+  return cuda_fail(cudaFuncSetAttribute(commit_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxReq * kSmemPerReq),
                    "commit_kernel shared-memory attribute");
 }
 
@@ -174,9 +182,11 @@ int launch_commit(lr_plan *p, const uint8_t *verdict, const int32_t *n_accept, i
     set_error("lr_commit: more than %d requests in one pass", kMaxReq);
     return LR_EUNSUPPORTED;
   }
-  int grid = (d.n_page_slots + 511) / 512;
-  grid = grid < 1 ? 1 : (grid > 64 ? 64 : grid);
-  size_t smem = (size_t)d.n_req * 16;
+  // every CTA repeats the per-request phase, so few CTAs when there are many requests
+  int grid = (d.n_page_slots + kThreads - 1) / kThreads;
+  const int cap = d.n_req <= 64 ? 148 : (d.n_req <= 512 ? 32 : 8);
+  grid = grid < 1 ? 1 : (grid > cap ? cap : grid);
+  size_t smem = (size_t)d.n_req * kSmemPerReq;
   commit_kernel<<<grid, kThreads, smem, s>>>(d, verdict, n_accept, n_steps, survivor, committed,
                                               keep_off, keep_pages, keep_valid, free_off, free_pages);
   p->ctx->launches++;

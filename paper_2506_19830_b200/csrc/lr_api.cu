@@ -98,7 +98,7 @@ static int validate_batch(const lr_batch *b) {
 struct Layout {
   Image img;
   size_t o_req_span_off, o_span_len, o_span_slot, o_br_req, o_br_depth, o_br_own_len, o_br_own_slot, o_br_n_draft, o_cu_q,
-      o_cu_draft, o_page_ids, o_req_br_off, o_span_req, o_status;
+      o_cu_draft, o_page_ids, o_req_br_off, o_span_req, o_status, o_slot_item, o_chain_pg, o_chain_tok, o_tail_pg;
   std::vector<int32_t> cu_draft;
   TcHostPlan tc;
   size_t image_bytes, total_bytes;
@@ -134,6 +134,29 @@ static int build_layout(const lr_ctx *ctx, const lr_batch *b, Layout &L) {
   L.o_page_ids = g.add(b->page_ids, I * b->n_page_slots);
   L.o_req_br_off = g.add(req_br_off.data(), I * (b->n_req + 1));
   L.o_span_req = g.add(span_req.data(), I * b->n_span);
+  {
+    std::vector<int32_t> slot_item((size_t)b->n_page_slots, -1), chain_pg((size_t)b->n_span + b->n_req, 0),
+        chain_tok((size_t)b->n_span + b->n_req, 0), tail_pg((size_t)b->n_branch + b->n_req, 0);
+    for (int r = 0; r < b->n_req; ++r) {
+      const int s0 = b->req_span_off[r], s1 = b->req_span_off[r + 1], base = s0 + r;
+      for (int s = s0; s < s1; ++s) {
+        const int npg = pages_of(b->span_len[s]);
+        chain_pg[base + (s - s0) + 1] = chain_pg[base + (s - s0)] + npg;
+        chain_tok[base + (s - s0) + 1] = chain_tok[base + (s - s0)] + b->span_len[s];
+        for (int k = 0; k < npg; ++k) slot_item[b->span_slot[s] + k] = s;
+      }
+      const int b0 = req_br_off[r], b1 = req_br_off[r + 1], tb = b0 + r;
+      for (int i = b0; i < b1; ++i) {
+        const int npg = pages_of(b->br_own_len[i]);
+        tail_pg[tb + (i - b0) + 1] = tail_pg[tb + (i - b0)] + npg;
+        for (int k = 0; k < npg; ++k) slot_item[b->br_own_slot[i] + k] = b->n_span + i;
+      }
+    }
+    L.o_slot_item = g.add(slot_item.data(), I * slot_item.size());
+    L.o_chain_pg = g.add(chain_pg.data(), I * chain_pg.size());
+    L.o_chain_tok = g.add(chain_tok.data(), I * chain_tok.size());
+    L.o_tail_pg = g.add(tail_pg.data(), I * tail_pg.size());
+  }
   int32_t zero2[2] = {0, 0};
   L.o_status = g.add(zero2, sizeof(zero2));
   L.cu_draft = cu_draft;
@@ -270,6 +293,10 @@ extern "C" int lr_plan_create(lr_ctx *ctx, const lr_batch *b, void *ws, size_t w
   d.page_ids = at(L.o_page_ids);
   d.req_br_off = at(L.o_req_br_off);
   d.span_req = at(L.o_span_req);
+  d.slot_item = at(L.o_slot_item);
+  d.chain_pg = at(L.o_chain_pg);
+  d.chain_tok = at(L.o_chain_tok);
+  d.tail_pg = at(L.o_tail_pg);
   d.status = reinterpret_cast<int32_t *>(base + L.o_status);
   d.n_req = b->n_req;
   d.n_branch = b->n_branch;

@@ -28,6 +28,13 @@ struct DevBatch {
   const int32_t *cu_q, *cu_draft, *page_ids;
   const int32_t *req_br_off;  // [n_req+1] branch range of each request
   const int32_t *span_req;    // [n_span] owning request of each span
+  // commit tables.  Request r's chain prefix sums start at index req_span_off[r] + r and have
+  // gamma_r + 2 entries: entry c = pages (tokens) of spans 0..c-1.  Its tail prefix sums start at
+  // req_br_off[r] + r: entry k = pages of the tails of its first k branches.
+  const int32_t *slot_item;   // [n_page_slots] owning span, or n_span + owning branch, or -1
+  const int32_t *chain_pg;    // [n_span + n_req]
+  const int32_t *chain_tok;   // [n_span + n_req]
+  const int32_t *tail_pg;     // [n_branch + n_req]
   int32_t n_req, n_branch, n_span, n_page_slots, n_q_rows;
   int32_t n_q_heads, n_kv_heads, head_dim, group;
   int64_t n_pool_pages;
