@@ -20,20 +20,21 @@
 // unnormalised O) and a small second kernel merges the partials of an M-tile in
 // a fixed order.
 //
-// One CTA = 11 warps:
-//   warp 0      TMA producer: the Q tiles of a piece (3-D boxes: 64 channels x G
+// One CTA = 12 warps in three warpgroups (registers are moved from the service warps to the
+// softmax warpgroups with setmaxnreg):
+//   warp 8      TMA producer: the Q tiles of a piece (3-D boxes: 64 channels x G
 //               heads x T tokens, so that the rows land packed) and, per tile,
 //               16 + 16 bulk tensor copies (one per page and 64-channel half, K
 //               and V) into a 5-stage ring of 32 KB buffers, all in the
 //               128-byte-swizzled layout the MMA descriptors read.  No multicast.
-//   warps 1, 2  MMA issuers of stream 0 and 1: tcgen05.mma (M=128, N=128, K=16,
+//   warps 9, 10 MMA issuers of stream 0 and 1 (warp 11 idles): tcgen05.mma (M=128, N=128, K=16,
 //               bf16 -> fp32) for S = Q K^T (both operands in shared memory) and
 //               O += P V (P read from tensor memory, V from shared memory as the
 //               N-major operand).  Issue blocks while the tensor pipe is full, so
 //               one issuer per stream lets the waits of one overlap the MMAs of
 //               the other.
-//   warps 3-6   softmax of stream 0, one thread per query row: tcgen05.ld gives a
-//   warps 7-10  softmax of stream 1  thread its whole row of S in registers, so
+//   warps 0-3   softmax of stream 0, one thread per query row: tcgen05.ld gives a
+//   warps 4-7   softmax of stream 1  thread its whole row of S in registers, so
 //               row max and row sum need no cross-lane traffic.  One sweep:
 //               max (3-input max), lazy rescale of O in tensor memory only when
 //               the maximum grew by more than 2^8, exp2 with packed fp32 FMA/ADD,
@@ -65,16 +66,17 @@ constexpr int kD = 128;
 constexpr int kStages = 5;
 constexpr int kTileBytes = 32768;  // [2 halves of 64 channels][128 keys or rows][128 B]
 constexpr int kHalfBytes = 16384;
-constexpr int kThreads = 352;
+constexpr int kThreads = 384;
 constexpr int kPagesPerTile = 8;
 constexpr uint64_t kWaitLimitNs = 1000ull * 1000ull * 1000ull;  // one second per wait, measured on the global timer
 constexpr uint64_t kDrainLimitNs = 50ull * 1000ull * 1000ull;
-constexpr float kRescaleThreshold = 8.0f;  // log2 units: P stays below 2^8
+constexpr float kRescaleThreshold = 8.0f;  // log2 units: the reference exponent follows the row maximum within 2^8
+constexpr float kRedoThreshold = 64.0f;    // log2 units: beyond this a tile is redone with its own maximum as reference
 
 struct __align__(8) Ctrl {
   uint64_t kv_full[kStages], kv_empty[kStages];
   uint64_t q_full, q_empty;
-  uint64_t s_full[2], p_full[2], o_done[2];
+  uint64_t s_full[2], p_half[2], p_full[2], o_done[2], turn[2];
   uint64_t epi_done, stagger, drain[2];
   uint32_t tmem_base;
   int abort_flag;
@@ -341,6 +343,34 @@ __device__ __forceinline__ float exp_half(const uint32_t (&v)[64], uint32_t (&pk
   return acc0.x + acc0.y;
 }
 
+// exp_half on v, and beside it (in the shadow of the MUFU) the maximum of the raw scores of v and w
+__device__ __forceinline__ float exp_half_max(const uint32_t (&v)[64], const uint32_t (&w)[64], uint32_t (&pk)[32], float scale_log2,
+                                              float neg_m, float &raw_max) {
+  const float2 sc = make_float2(scale_log2, scale_log2), nm = make_float2(neg_m, neg_m);
+  float2 acc0 = make_float2(0.f, 0.f), acc1 = make_float2(0.f, 0.f);
+  float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
+#pragma unroll
+  for (int i = 0; i < 64; i += 4) {
+    float2 y0 = ffma2(make_float2(bits_f(v[i]), bits_f(v[i + 1])), sc, nm);
+    float2 y1 = ffma2(make_float2(bits_f(v[i + 2]), bits_f(v[i + 3])), sc, nm);
+    m0 = max3(m0, bits_f(v[i]), bits_f(v[i + 1]));
+    m1 = max3(m1, bits_f(v[i + 2]), bits_f(v[i + 3]));
+    y0.x = ex2(y0.x);
+    y0.y = ex2(y0.y);
+    m2 = max3(m2, bits_f(w[i]), bits_f(w[i + 1]));
+    m3 = max3(m3, bits_f(w[i + 2]), bits_f(w[i + 3]));
+    y1.x = ex2(y1.x);
+    y1.y = ex2(y1.y);
+    acc0 = fadd2(acc0, y0);
+    acc1 = fadd2(acc1, y1);
+    pk[i >> 1] = pack_bf16(y0.x, y0.y);
+    pk[(i >> 1) + 1] = pack_bf16(y1.x, y1.y);
+  }
+  raw_max = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
+  acc0 = fadd2(acc0, acc1);
+  return acc0.x + acc0.y;
+}
+
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map,
                const __grid_constant__ CUtensorMap q_map, DevBatch d, DevTcPlan tc, uint16_t *__restrict__ out,
@@ -370,7 +400,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant_
     mbar_init(&ctrl->q_empty, 2);
     for (int s = 0; s < 2; ++s) {
       mbar_init(&ctrl->s_full[s], 1);
+      mbar_init(&ctrl->p_half[s], 128);
       mbar_init(&ctrl->p_full[s], 128);
+      mbar_init(&ctrl->turn[s], 1);
       mbar_init(&ctrl->o_done[s], 1);
       mbar_init(&ctrl->drain[s], 1);
     }
@@ -379,7 +411,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant_
     ctrl->abort_flag = 0;
     fence_barrier_init();
   }
-  if (warp == 1) {
+  if (warp == 9) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctrl->tmem_base)), "r"(512u)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -396,7 +428,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant_
   const int T = tc.tokens_per_mtile;
   const int G = d.group;
 
-  if (warp == 0) {
+  if (warp >= 8) {
+   // service warpgroup: needs few registers; the softmax threads hold a whole row of scores in theirs
+   asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
+   if (warp == 8) {
     // ======================= TMA producer ==========================================
     uint32_t ring = 0, q_count = 0;
     bool ok = true;
@@ -463,13 +498,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant_
           if (global_ns() - t0 > kDrainLimitNs) break;
       }
     }
-  } else if (warp <= 2) {
+   } else if (warp == 9 || warp == 10) {
     // ======================= MMA issuer of stream s ====================================
     // Both issuers walk every ring position of a piece in order: a position this stream uses is
     // consumed by its MMAs (released by a tcgen05.commit), one it does not use (the other
     // stream's tiles in the even/odd split) is released with a plain arrive once it has landed.
     // So neither issuer nor the producer can get a whole ring ahead of the other.
-    const int s = warp - 1;
+    const int s = warp - 9;
     uint32_t ring_base = 0, waited = 0, p_cnt = 0, pc_idx = 0;
     bool ok = true;
     const uint32_t q_addr = smem_u32(q_smem), kv_addr = smem_u32(kv_smem);
@@ -486,17 +521,24 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant_
           mma_ss(s_tmem, a + (uint64_t)(h * (kHalfBytes >> 4) + kk * 2), b + (uint64_t)(h * (kHalfBytes >> 4) + kk * 2), kIdescQK,
                  (h | kk) != 0);
     };
-    auto issue_pv = [&](uint32_t stage, bool acc) {  // O_s (+)= P_s V
+    auto issue_pv = [&](uint32_t stage, int half, bool acc) {  // O_s (+)= P_s V over 64 of the 128 keys
       const uint64_t b = vdesc0 + (uint64_t)(stage * (kTileBytes >> 4));
 #pragma unroll
-      for (int ks = 0; ks < 8; ++ks) mma_ts(o_tmem, s_tmem + ks * 8, b + (uint64_t)(ks * (2048 >> 4)), kIdescPV, acc || ks != 0);
+      for (int k4 = 0; k4 < 4; ++k4) {
+        const int ks = half * 4 + k4;
+        mma_ts(o_tmem, s_tmem + ks * 8, b + (uint64_t)(ks * (2048 >> 4)), kIdescPV, acc || ks != 0);
+      }
     };
+    // Batches (the PV of a unit and the QK of the next) of the two streams are issued in turns --
+    // 0, 1, 0, 1, ... in the order of the units -- so that the streams stay half a period apart.
+    uint32_t c_mine = 0, c_other = 0;  // batches issued before this piece by this issuer / the other one
     for (int pc = piece0; pc < piece1 && ok; ++pc, ++pc_idx) {
       const TcPiece pi = tc.pieces[pc];
       const TcReq rq = tc.reqs[pi.req];
       const int n = pi.tile_end - pi.tile_begin, mode = pi.n_mt;
       const RingOrder ord(n, mode);
       const int my_units = mode == 2 ? n : (n - s + 1) / 2;
+      const int other_units = mode == 2 ? n : (n - (1 - s) + 1) / 2;
       const int m_tile = mode == 2 ? s : 0;
       // waits, in ring order, until absolute ring position `pos` has landed; positions on the way
       // belong to the other stream and are released here
@@ -527,8 +569,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant_
           issue_qk(m_tile, pos % kStages);
           tc_commit(&ctrl->s_full[s]);
           release(pos);
+          if (my_units == 1) tc_commit(&ctrl->q_empty);  // last QK of the piece: this stream is done with the Q buffers
         }
         __syncwarp();
+      } else if (lane == 0) {
+        mbar_arrive(&ctrl->q_empty);
       }
       for (int j = 0; j < my_units && ok; ++j) {
         const int t = mode == 2 ? j : 2 * j + s;
@@ -561,22 +606,39 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant_
           ok = wait_bar(&ctrl->epi_done, (pc_idx - 1) & 1u, ctrl, d.status, 223);
           if (!ok) break;
         }
+        {
+          // my turn: stream 0 goes after stream 1's previous batch, stream 1 after stream 0's batch of the same unit
+          const uint32_t want = c_other + (uint32_t)(s == 0 ? min(j, other_units) : j + 1);
+          if (want > 0) {
+            ok = wait_bar(&ctrl->turn[s], (want - 1) & 1u, ctrl, d.status, 228);
+            if (!ok) break;
+          }
+        }
+        ok = wait_bar(&ctrl->p_half[s], p_cnt & 1u, ctrl, d.status, 229);
+        if (!ok) break;
+        tc_fence_after();
+        if (lane == 0) issue_pv(sV, 0, j > 0);
+        __syncwarp();
         ok = wait_bar(&ctrl->p_full[s], p_cnt & 1u, ctrl, d.status, 224 + s);
         ++p_cnt;
         if (!ok) break;
         tc_fence_after();
         if (lane == 0) {
-          issue_pv(sV, j > 0);
+          issue_pv(sV, 1, true);
           tc_commit(&ctrl->o_done[s]);
           release(pos_v);
           if (has_next) {
             issue_qk(m_tile, pos_k % kStages);
             tc_commit(&ctrl->s_full[s]);
             release(pos_k);
+            if (j + 2 == my_units) tc_commit(&ctrl->q_empty);  // last QK of the piece
           }
+          mbar_arrive(&ctrl->turn[1 - s]);
         }
         __syncwarp();
       }
+      c_mine += (uint32_t)my_units;
+      c_other += (uint32_t)other_units;
       if (!ok) break;
       // positions of the piece this stream never touched (the tail of the other stream's tiles)
       ring_base += 2u * (uint32_t)n;
@@ -585,8 +647,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant_
         if (!ok) break;
         if (lane == 0) mbar_arrive(&ctrl->kv_empty[(ring_base - 1) % kStages]);
       }
-      if (lane == 0) tc_commit(&ctrl->q_empty);  // every MMA of this stream retired: its reads of the Q buffers are done
-      __syncwarp();
     }
     if (!ok && lane == 0) {
       // let every MMA already issued retire before tensor memory is released
@@ -596,9 +656,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant_
         if (global_ns() - t0 > kDrainLimitNs) break;
     }
     __syncwarp();
+   }
   } else {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
     // ======================= softmax warpgroups ======================================
-    const int s = (warp - 3) >> 2;                 // stream
+    const int s = warp >> 2;                       // stream
     const int quarter = warp & 3;                  // tensor-memory lane quarter this warp may access
     const int r = quarter * 32 + lane;             // row within the M-tile
     const uint32_t lane_base = tmem + ((uint32_t)(quarter * 32) << 16);
@@ -612,7 +674,20 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant_
       const int my_units = mode == 2 ? n : (n - s + 1) / 2;
       if (ok && my_units > 0) {
         const RowInfo ri = row_info(d, tc, rq, T, mode == 2 ? pi.mtile0 + s : pi.mtile0, r, pi.kv_head);
-        float m_used = -INFINITY, l = 0.f;
+        float m_used = -INFINITY, l = 0.f, m_new = 0.f;
+        bool pend = false;
+        auto rescale_o = [&](float alpha) {
+#pragma unroll
+          for (int ch = 0; ch < 4; ++ch) {
+            uint32_t o[32];
+            tmem_ld32(o_addr + ch * 32, o);
+            tc_wait_ld();
+#pragma unroll
+            for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(bits_f(o[c]) * alpha);
+            tmem_st32(o_addr + ch * 32, o);
+          }
+          tc_wait_st();
+        };
         for (int j = 0; j < my_units; ++j) {
           const int t = pi.tile_begin + (mode == 2 ? j : 2 * j + s);
           ok = wait_bar(&ctrl->s_full[s], s_cnt & 1u, ctrl, d.status, 230 + s);
@@ -635,32 +710,53 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant_
             mask_half(va, n_ok);
             mask_half(vb, n_ok + 4);
           }
-          const float mx = fmaxf(max_half(va), max_half(vb)) * scale_log2;
-          // lazy rescale: only when the maximum grew by more than the threshold
-          const bool grow = mx > m_used + kRescaleThreshold;
-          if (__any_sync(0xFFFFFFFFu, grow)) {
-            const float alpha = grow ? ex2(m_used - mx) : 1.0f;
-            if (grow) {
+          // A growth of the maximum noticed in the previous unit is applied now: the PV product of that
+          // unit has retired (its commit precedes s_full's), so O may be rescaled.
+          if (__any_sync(0xFFFFFFFFu, pend)) {
+            const float alpha = pend ? ex2(m_used - m_new) : 1.0f;
+            if (pend) {
               l *= alpha;
-              m_used = mx;
+              m_used = m_new;
+              pend = false;
             }
-            if (j > 0) {  // the PV product of this stream's previous unit has retired (its commit precedes s_full's)
-#pragma unroll
-              for (int ch = 0; ch < 4; ++ch) {
-                uint32_t o[32];
-                tmem_ld32(o_addr + ch * 32, o);
-                tc_wait_ld();
-#pragma unroll
-                for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(bits_f(o[c]) * alpha);
-                tmem_st32(o_addr + ch * 32, o);
+            rescale_o(alpha);
+          }
+          uint32_t pk[32];
+          float sum_a = 0.f, mx;
+          // Fast path: exponentials against the running reference exponent; the row maximum is computed
+          // beside them and only checked afterwards.
+          bool fast = __all_sync(0xFFFFFFFFu, m_used > -INFINITY);
+          if (fast) {
+            float raw;
+            sum_a = exp_half_max(va, vb, pk, scale_log2, -m_used, raw);
+            mx = raw * scale_log2;
+            if (__any_sync(0xFFFFFFFFu, mx > m_used + kRedoThreshold)) fast = false;  // could overflow: redo exactly
+          } else {
+            mx = fmaxf(max_half(va), max_half(vb)) * scale_log2;
+          }
+          if (!fast) {
+            // Exact path (first unit of a stream, rows that have seen no key yet, a jump of the scores):
+            // adopt the row maximum before the exponentials.
+            const bool grow = mx > m_used + kRescaleThreshold;
+            if (__any_sync(0xFFFFFFFFu, grow)) {
+              const float alpha = grow ? ex2(m_used - mx) : 1.0f;
+              if (grow) {
+                l *= alpha;
+                m_used = mx;
               }
-              tc_wait_st();
+              if (j > 0) rescale_o(alpha);
             }
+            sum_a = exp_half(va, pk, scale_log2, (m_used == -INFINITY) ? 0.f : -m_used);
+          } else if (mx > m_used + kRescaleThreshold) {
+            pend = true;
+            m_new = mx;
           }
           const float neg_m = (m_used == -INFINITY) ? 0.f : -m_used;
-          uint32_t pk[32];
-          l += exp_half(va, pk, scale_log2, neg_m);
+          l += sum_a;
           tmem_st32(s_addr, pk);
+          tc_wait_st();
+          tc_fence_before();
+          mbar_arrive(&ctrl->p_half[s]);  // the PV product may start on the first 64 keys
           l += exp_half(vb, pk, scale_log2, neg_m);
           tmem_st32(s_addr + 32, pk);
           tc_wait_st();
@@ -718,7 +814,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant_
 
   tc_fence_before();
   __syncthreads();
-  if (warp == 1) {
+  if (warp == 9) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
   }
@@ -919,9 +1015,12 @@ int tc_build_host_plan(const lr_ctx *ctx, const lr_batch *b, const int32_t *req_
   if (grps.empty()) return LR_OK;
   // Cut the weighted tile sequence into n_cta contiguous ranges of equal weight: a tile belongs to the
   // CTA whose weight interval [total*c/n, total*(c+1)/n) holds the tile's start position.
+  // The start of a group inside a CTA's range (epilogue, Q reload, pipeline ramp) is charged like
+  // kPieceStartTiles tiles, so such a CTA gets fewer tiles.
+  constexpr int kPieceStartTiles = 4;
   int64_t total_w = 0, total_tiles = 0;
   for (const Grp &g : grps) {
-    total_w += (int64_t)g.n_tiles * g.weight;
+    total_w += (int64_t)(g.n_tiles + kPieceStartTiles) * g.weight;
     total_tiles += g.n_tiles;
   }
   const int n_cta = (int)std::min<int64_t>(ctx->sm_count, std::max<int64_t>(1, total_tiles / 2));
@@ -933,6 +1032,7 @@ int tc_build_host_plan(const lr_ctx *ctx, const lr_batch *b, const int32_t *req_
   for (size_t gi = 0; gi < grps.size(); ++gi) {
     Grp &g = grps[gi];
     g.first_piece = (int)pieces.size();
+    w_pos += (int64_t)kPieceStartTiles * g.weight;
     for (int t = 0; t < g.n_tiles; ++t, w_pos += g.weight) {
       while (cta + 1 < n_cta && w_pos >= total_w * (cta + 1) / n_cta) {
         ++cta;
