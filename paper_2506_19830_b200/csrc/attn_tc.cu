@@ -76,8 +76,8 @@ constexpr float kRedoThreshold = 64.0f;    // log2 units: beyond this a tile is 
 struct __align__(8) Ctrl {
   uint64_t kv_full[kStages], kv_empty[kStages];
   uint64_t q_full, q_empty;
-  uint64_t s_full[2], p_half[2], p_full[2], o_done[2], turn[2];
-  uint64_t epi_done, stagger, drain[2];
+  uint64_t s_full[2][2], p_full[2][2], o_done[2];  // [stream][half]
+  uint64_t epi_done, drain[2];
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -147,9 +147,11 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t addr, uint32_t lbo_bytes,
   return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) | ((uint64_t)(sbo_bytes >> 4) << 32) |
          (1ull << 46) | (2ull << 61);
 }
-// Instruction descriptor: D fp32, A and B bf16, M = 128, N = 128; bit 16 selects an N-major B operand.
-constexpr uint32_t kIdescQK = (1u << 4) | (1u << 7) | (1u << 10) | (16u << 17) | (8u << 24);
-constexpr uint32_t kIdescPV = kIdescQK | (1u << 16);
+// Instruction descriptors: D fp32, A and B bf16, M = 128 (bits 24-28 = M/16), N in bits 17-22 (= N/8).
+// QK: N = 64 keys of a half-tile, both operands K-major.  PV: N = 128 channels, bit 16 selects the N-major B operand.
+constexpr uint32_t kIdescBase = (1u << 4) | (1u << 7) | (1u << 10) | (8u << 24);
+constexpr uint32_t kIdescQK = kIdescBase | ((64u >> 3) << 17);
+constexpr uint32_t kIdescPV = kIdescBase | ((128u >> 3) << 17) | (1u << 16);
 
 __device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
   asm volatile(
@@ -343,22 +345,20 @@ __device__ __forceinline__ float exp_half(const uint32_t (&v)[64], uint32_t (&pk
   return acc0.x + acc0.y;
 }
 
-// exp_half on v, and beside it (in the shadow of the MUFU) the maximum of the raw scores of v and w
-__device__ __forceinline__ float exp_half_max(const uint32_t (&v)[64], const uint32_t (&w)[64], uint32_t (&pk)[32], float scale_log2,
-                                              float neg_m, float &raw_max) {
+// exp_half on v, and beside it (in the shadow of the MUFU) the maximum of the raw scores
+__device__ __forceinline__ float exp_half_max(const uint32_t (&v)[64], uint32_t (&pk)[32], float scale_log2, float neg_m,
+                                              float &raw_max) {
   const float2 sc = make_float2(scale_log2, scale_log2), nm = make_float2(neg_m, neg_m);
   float2 acc0 = make_float2(0.f, 0.f), acc1 = make_float2(0.f, 0.f);
-  float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
+  float m0 = -INFINITY, m1 = -INFINITY;
 #pragma unroll
   for (int i = 0; i < 64; i += 4) {
     float2 y0 = ffma2(make_float2(bits_f(v[i]), bits_f(v[i + 1])), sc, nm);
     float2 y1 = ffma2(make_float2(bits_f(v[i + 2]), bits_f(v[i + 3])), sc, nm);
     m0 = max3(m0, bits_f(v[i]), bits_f(v[i + 1]));
-    m1 = max3(m1, bits_f(v[i + 2]), bits_f(v[i + 3]));
     y0.x = ex2(y0.x);
     y0.y = ex2(y0.y);
-    m2 = max3(m2, bits_f(w[i]), bits_f(w[i + 1]));
-    m3 = max3(m3, bits_f(w[i + 2]), bits_f(w[i + 3]));
+    m1 = max3(m1, bits_f(v[i + 2]), bits_f(v[i + 3]));
     y1.x = ex2(y1.x);
     y1.y = ex2(y1.y);
     acc0 = fadd2(acc0, y0);
@@ -366,7 +366,7 @@ __device__ __forceinline__ float exp_half_max(const uint32_t (&v)[64], const uin
     pk[i >> 1] = pack_bf16(y0.x, y0.y);
     pk[(i >> 1) + 1] = pack_bf16(y1.x, y1.y);
   }
-  raw_max = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
+  raw_max = fmaxf(m0, m1);
   acc0 = fadd2(acc0, acc1);
   return acc0.x + acc0.y;
 }
@@ -399,15 +399,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant_
     mbar_init(&ctrl->q_full, 1);
     mbar_init(&ctrl->q_empty, 2);
     for (int s = 0; s < 2; ++s) {
-      mbar_init(&ctrl->s_full[s], 1);
-      mbar_init(&ctrl->p_half[s], 128);
-      mbar_init(&ctrl->p_full[s], 128);
-      mbar_init(&ctrl->turn[s], 1);
+      for (int h = 0; h < 2; ++h) {
+        mbar_init(&ctrl->s_full[s][h], 1);
+        mbar_init(&ctrl->p_full[s][h], 128);
+      }
       mbar_init(&ctrl->o_done[s], 1);
       mbar_init(&ctrl->drain[s], 1);
     }
     mbar_init(&ctrl->epi_done, 256);
-    mbar_init(&ctrl->stagger, 128);
     ctrl->abort_flag = 0;
     fence_barrier_init();
   }
@@ -512,33 +511,28 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant_
     // Descriptors differ from a base only in the start-address field (units of 16 bytes).
     const uint64_t qdesc0 = make_desc(q_addr, 16, 1024), kdesc0 = make_desc(kv_addr, 16, 1024),
                    vdesc0 = make_desc(kv_addr, kHalfBytes, 1024);
-    auto issue_qk = [&](int m, uint32_t stage) {  // S_s = Q_m K^T
-      const uint64_t a = qdesc0 + (uint64_t)(m * (kTileBytes >> 4)), b = kdesc0 + (uint64_t)(stage * (kTileBytes >> 4));
+    auto issue_qk = [&](int m, uint32_t stage, int half) {  // S_s[half] = Q_m K^T over 64 of the 128 keys
+      const uint64_t a = qdesc0 + (uint64_t)(m * (kTileBytes >> 4)),
+                     b = kdesc0 + (uint64_t)(stage * (kTileBytes >> 4) + half * (64 * 128 >> 4));
 #pragma unroll
       for (int h = 0; h < 2; ++h)
 #pragma unroll
         for (int kk = 0; kk < 4; ++kk)
-          mma_ss(s_tmem, a + (uint64_t)(h * (kHalfBytes >> 4) + kk * 2), b + (uint64_t)(h * (kHalfBytes >> 4) + kk * 2), kIdescQK,
-                 (h | kk) != 0);
+          mma_ss(s_tmem + half * 64, a + (uint64_t)(h * (kHalfBytes >> 4) + kk * 2), b + (uint64_t)(h * (kHalfBytes >> 4) + kk * 2),
+                 kIdescQK, (h | kk) != 0);
     };
-    auto issue_pv = [&](uint32_t stage, int half, bool acc) {  // O_s (+)= P_s V over 64 of the 128 keys
-      const uint64_t b = vdesc0 + (uint64_t)(stage * (kTileBytes >> 4));
+    auto issue_pv = [&](uint32_t stage, int half, bool acc) {  // O_s (+)= P_s[half] V over 64 of the 128 keys
+      const uint64_t b = vdesc0 + (uint64_t)(stage * (kTileBytes >> 4) + half * (4 * 2048 >> 4));
 #pragma unroll
-      for (int k4 = 0; k4 < 4; ++k4) {
-        const int ks = half * 4 + k4;
-        mma_ts(o_tmem, s_tmem + ks * 8, b + (uint64_t)(ks * (2048 >> 4)), kIdescPV, acc || ks != 0);
-      }
+      for (int k4 = 0; k4 < 4; ++k4)
+        mma_ts(o_tmem, s_tmem + half * 64 + k4 * 8, b + (uint64_t)(k4 * (2048 >> 4)), kIdescPV, acc || k4 != 0);
     };
-    // Batches (the PV of a unit and the QK of the next) of the two streams are issued in turns --
-    // 0, 1, 0, 1, ... in the order of the units -- so that the streams stay half a period apart.
-    uint32_t c_mine = 0, c_other = 0;  // batches issued before this piece by this issuer / the other one
     for (int pc = piece0; pc < piece1 && ok; ++pc, ++pc_idx) {
       const TcPiece pi = tc.pieces[pc];
       const TcReq rq = tc.reqs[pi.req];
       const int n = pi.tile_end - pi.tile_begin, mode = pi.n_mt;
       const RingOrder ord(n, mode);
       const int my_units = mode == 2 ? n : (n - s + 1) / 2;
-      const int other_units = mode == 2 ? n : (n - (1 - s) + 1) / 2;
       const int m_tile = mode == 2 ? s : 0;
       // waits, in ring order, until absolute ring position `pos` has landed; positions on the way
       // belong to the other stream and are released here
@@ -555,19 +549,15 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant_
       ok = wait_bar(&ctrl->q_full, pc_idx & 1u, ctrl, d.status, 220);
       if (!ok) break;
       if (my_units > 0) {
-        if (s == 1) {
-          // Start half a period behind stream 0 (after its first softmax), so that the two streams use
-          // the MUFU and the tensor pipe in turns instead of both at once.
-          ok = wait_bar(&ctrl->stagger, pc_idx & 1u, ctrl, d.status, 219);
-          if (!ok) break;
-        }
         const uint32_t pos = ring_base + ord.pos_k(mode == 2 ? 0 : s);
         ok = need(pos, 221);
         if (!ok) break;
         tc_fence_after();
         if (lane == 0) {
-          issue_qk(m_tile, pos % kStages);
-          tc_commit(&ctrl->s_full[s]);
+          issue_qk(m_tile, pos % kStages, 0);
+          tc_commit(&ctrl->s_full[s][0]);
+          issue_qk(m_tile, pos % kStages, 1);
+          tc_commit(&ctrl->s_full[s][1]);
           release(pos);
           if (my_units == 1) tc_commit(&ctrl->q_empty);  // last QK of the piece: this stream is done with the Q buffers
         }
@@ -606,39 +596,29 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant_
           ok = wait_bar(&ctrl->epi_done, (pc_idx - 1) & 1u, ctrl, d.status, 223);
           if (!ok) break;
         }
-        {
-          // my turn: stream 0 goes after stream 1's previous batch, stream 1 after stream 0's batch of the same unit
-          const uint32_t want = c_other + (uint32_t)(s == 0 ? min(j, other_units) : j + 1);
-          if (want > 0) {
-            ok = wait_bar(&ctrl->turn[s], (want - 1) & 1u, ctrl, d.status, 228);
-            if (!ok) break;
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+          // P of this half is in place: O += P V, then the buffer takes the scores of the next tile's half
+          ok = wait_bar(&ctrl->p_full[s][half], p_cnt & 1u, ctrl, d.status, 224 + s);
+          if (!ok) break;
+          tc_fence_after();
+          if (lane == 0) {
+            issue_pv(sV, half, (j | half) != 0);
+            tc_commit(&ctrl->o_done[s]);
+            if (half == 1) release(pos_v);
+            if (has_next) {
+              issue_qk(m_tile, pos_k % kStages, half);
+              tc_commit(&ctrl->s_full[s][half]);
+              if (half == 1) {
+                release(pos_k);
+                if (j + 2 == my_units) tc_commit(&ctrl->q_empty);  // last QK of the piece
+              }
+            }
           }
+          __syncwarp();
         }
-        ok = wait_bar(&ctrl->p_half[s], p_cnt & 1u, ctrl, d.status, 229);
-        if (!ok) break;
-        tc_fence_after();
-        if (lane == 0) issue_pv(sV, 0, j > 0);
-        __syncwarp();
-        ok = wait_bar(&ctrl->p_full[s], p_cnt & 1u, ctrl, d.status, 224 + s);
         ++p_cnt;
-        if (!ok) break;
-        tc_fence_after();
-        if (lane == 0) {
-          issue_pv(sV, 1, true);
-          tc_commit(&ctrl->o_done[s]);
-          release(pos_v);
-          if (has_next) {
-            issue_qk(m_tile, pos_k % kStages);
-            tc_commit(&ctrl->s_full[s]);
-            release(pos_k);
-            if (j + 2 == my_units) tc_commit(&ctrl->q_empty);  // last QK of the piece
-          }
-          mbar_arrive(&ctrl->turn[1 - s]);
-        }
-        __syncwarp();
       }
-      c_mine += (uint32_t)my_units;
-      c_other += (uint32_t)other_units;
       if (!ok) break;
       // positions of the piece this stream never touched (the tail of the other stream's tiles)
       ring_base += 2u * (uint32_t)n;
@@ -665,7 +645,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant_
     const int r = quarter * 32 + lane;             // row within the M-tile
     const uint32_t lane_base = tmem + ((uint32_t)(quarter * 32) << 16);
     const uint32_t s_addr = lane_base + s * 128, o_addr = lane_base + 256 + s * 128;
-    uint32_t s_cnt = 0, o_cnt = 0;
+    uint32_t s_cnt = 0, o_cnt = 0;  // tiles / half-units of this stream so far
     bool ok = true;
     for (int pc = piece0; pc < piece1; ++pc) {
       const TcPiece pi = tc.pieces[pc];
@@ -676,7 +656,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant_
         const RowInfo ri = row_info(d, tc, rq, T, mode == 2 ? pi.mtile0 + s : pi.mtile0, r, pi.kv_head);
         float m_used = -INFINITY, l = 0.f, m_new = 0.f;
         bool pend = false;
-        auto rescale_o = [&](float alpha) {
+        // O *= alpha.  The PV product of the previous half-unit must have retired first; the one before
+        // it has (its commit precedes the s_full this thread has just seen).
+        auto rescale_o = [&](float alpha, uint32_t done_needed) -> bool {
+          if (!wait_bar(&ctrl->o_done[s], (done_needed - 1) & 1u, ctrl, d.status, 235 + s)) return false;
+          tc_fence_after();
 #pragma unroll
           for (int ch = 0; ch < 4; ++ch) {
             uint32_t o[32];
@@ -687,19 +671,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant_
             tmem_st32(o_addr + ch * 32, o);
           }
           tc_wait_st();
+          return true;
         };
-        for (int j = 0; j < my_units; ++j) {
+        for (int j = 0; j < my_units && ok; ++j) {
           const int t = pi.tile_begin + (mode == 2 ? j : 2 * j + s);
-          ok = wait_bar(&ctrl->s_full[s], s_cnt & 1u, ctrl, d.status, 230 + s);
-          ++s_cnt;
-          if (!ok) break;
-          tc_fence_after();
-          uint32_t va[64], vb[64];
-          tmem_ld64(s_addr, va);
-          tmem_ld64(s_addr + 64, vb);
-          tc_wait_ld();
-          if (t >= rq.n_dense_tiles) {
-            int n_ok[kPagesPerTile];
+          const bool masked = t >= rq.n_dense_tiles;
+          int n_ok[kPagesPerTile];
+          if (masked) {
             const uint4 *mp = reinterpret_cast<const uint4 *>(tc.pages + rq.page_off + t * kPagesPerTile);
 #pragma unroll
             for (int jj = 0; jj < 4; ++jj) {
@@ -707,66 +685,81 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant_
               n_ok[2 * jj] = page_n_ok(w.y, ri);
               n_ok[2 * jj + 1] = page_n_ok(w.w, ri);
             }
-            mask_half(va, n_ok);
-            mask_half(vb, n_ok + 4);
           }
-          // A growth of the maximum noticed in the previous unit is applied now: the PV product of that
-          // unit has retired (its commit precedes s_full's), so O may be rescaled.
-          if (__any_sync(0xFFFFFFFFu, pend)) {
-            const float alpha = pend ? ex2(m_used - m_new) : 1.0f;
-            if (pend) {
-              l *= alpha;
-              m_used = m_new;
-              pend = false;
-            }
-            rescale_o(alpha);
-          }
-          uint32_t pk[32];
-          float sum_a = 0.f, mx;
-          // Fast path: exponentials against the running reference exponent; the row maximum is computed
-          // beside them and only checked afterwards.
-          bool fast = __all_sync(0xFFFFFFFFu, m_used > -INFINITY);
-          if (fast) {
-            float raw;
-            sum_a = exp_half_max(va, vb, pk, scale_log2, -m_used, raw);
-            mx = raw * scale_log2;
-            if (__any_sync(0xFFFFFFFFu, mx > m_used + kRedoThreshold)) fast = false;  // could overflow: redo exactly
-          } else {
-            mx = fmaxf(max_half(va), max_half(vb)) * scale_log2;
-          }
-          if (!fast) {
-            // Exact path (first unit of a stream, rows that have seen no key yet, a jump of the scores):
-            // adopt the row maximum before the exponentials.
-            const bool grow = mx > m_used + kRescaleThreshold;
-            if (__any_sync(0xFFFFFFFFu, grow)) {
-              const float alpha = grow ? ex2(m_used - mx) : 1.0f;
-              if (grow) {
+#pragma unroll
+          for (int half = 0; half < 2; ++half) {
+            const uint32_t sh_addr = s_addr + half * 64;
+            const uint32_t g = o_cnt + (uint32_t)(2 * j + half);  // half-units of this stream before this one
+            const bool first = (j | half) == 0;
+            ok = wait_bar(&ctrl->s_full[s][half], s_cnt & 1u, ctrl, d.status, 230 + s);
+            if (!ok) break;
+            tc_fence_after();
+            uint32_t v[64];
+            tmem_ld64(sh_addr, v);
+            tc_wait_ld();
+            if (masked) mask_half(v, n_ok + 4 * half);
+            // A growth of the maximum noticed in an earlier half-unit is applied now.
+            if (__any_sync(0xFFFFFFFFu, pend)) {
+              const float alpha = pend ? ex2(m_used - m_new) : 1.0f;
+              if (pend) {
                 l *= alpha;
-                m_used = mx;
+                m_used = m_new;
+                pend = false;
               }
-              if (j > 0) rescale_o(alpha);
+              ok = rescale_o(alpha, g);
+              if (!ok) break;
             }
-            sum_a = exp_half(va, pk, scale_log2, (m_used == -INFINITY) ? 0.f : -m_used);
-          } else if (mx > m_used + kRescaleThreshold) {
-            pend = true;
-            m_new = mx;
+            uint32_t pk[32];
+            float sum = 0.f, mx;
+            // Fast path: exponentials against the running reference exponent; the maximum of the 64 scores is
+            // computed beside them and only checked afterwards.
+            bool fast = __all_sync(0xFFFFFFFFu, m_used > -INFINITY);
+            if (fast) {
+              float raw;
+              sum = exp_half_max(v, pk, scale_log2, -m_used, raw);
+              mx = raw * scale_log2;
+              if (__any_sync(0xFFFFFFFFu, mx > m_used + kRedoThreshold)) fast = false;  // could overflow: redo exactly
+            } else {
+              mx = max_half(v) * scale_log2;
+            }
+            if (!fast) {
+              // Exact path (first half-unit of a stream, rows that have seen no key yet, a jump of the
+              // scores): adopt the maximum before the exponentials.
+              const bool grow = mx > m_used + kRescaleThreshold;
+              if (__any_sync(0xFFFFFFFFu, grow)) {
+                const float alpha = grow ? ex2(m_used - mx) : 1.0f;
+                if (grow) {
+                  l *= alpha;
+                  m_used = mx;
+                }
+                if (!first) {
+                  ok = rescale_o(alpha, g);
+                  if (!ok) break;
+                }
+              }
+              sum = exp_half(v, pk, scale_log2, (m_used == -INFINITY) ? 0.f : -m_used);
+            } else if (mx > m_used + kRescaleThreshold) {
+              pend = true;
+              m_new = mx;
+            }
+            l += sum;
+            tmem_st32(sh_addr, pk);
+            tc_wait_st();
+            tc_fence_before();
+            // Observe every completion of o_done in order (a parity wait must never fall two phases behind):
+            // the PV product of the previous half-unit has long retired by now.  Before the arrive below,
+            // because the PV product of this half-unit can only be issued after it.
+            if (g > 0) {
+              ok = wait_bar(&ctrl->o_done[s], (g - 1) & 1u, ctrl, d.status, 237 + s);
+              if (!ok) break;
+            }
+            mbar_arrive(&ctrl->p_full[s][half]);
           }
-          const float neg_m = (m_used == -INFINITY) ? 0.f : -m_used;
-          l += sum_a;
-          tmem_st32(s_addr, pk);
-          tc_wait_st();
-          tc_fence_before();
-          mbar_arrive(&ctrl->p_half[s]);  // the PV product may start on the first 64 keys
-          l += exp_half(vb, pk, scale_log2, neg_m);
-          tmem_st32(s_addr + 32, pk);
-          tc_wait_st();
-          tc_fence_before();
-          mbar_arrive(&ctrl->p_full[s]);
-          if (s == 0 && j == 0) mbar_arrive(&ctrl->stagger);
+          ++s_cnt;
         }
         if (ok) {
           // epilogue: wait for the last PV of this stream, then normalise and store
-          o_cnt += (uint32_t)my_units;
+          o_cnt += 2u * (uint32_t)my_units;
           ok = wait_bar(&ctrl->o_done[s], (o_cnt - 1) & 1u, ctrl, d.status, 240 + s);
         }
         if (ok) {
