@@ -429,6 +429,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant_
 
   if (warp >= 8) {
    // service warpgroup: needs few registers; the softmax threads hold a whole row of scores in theirs
+   // setmaxnreg.inc blocks until its request fits into what the CTA was launched with (168 registers x 384
+   // threads), so the totals after the moves must not exceed that: 72 x 128 + 216 x 256 = 168 x 384.
    asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
    if (warp == 8) {
     // ======================= TMA producer ==========================================
@@ -596,7 +598,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant_
           ok = wait_bar(&ctrl->epi_done, (pc_idx - 1) & 1u, ctrl, d.status, 223);
           if (!ok) break;
         }
-#pragma unroll
+#pragma unroll 1
         for (int half = 0; half < 2; ++half) {
           // P of this half is in place: O += P V, then the buffer takes the scores of the next tile's half
           ok = wait_bar(&ctrl->p_full[s][half], p_cnt & 1u, ctrl, d.status, 224 + s);
@@ -686,7 +688,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant_
               n_ok[2 * jj + 1] = page_n_ok(w.w, ri);
             }
           }
-#pragma unroll
+#pragma unroll 1  // one copy of the sweep: the unrolled pair was slower (instruction fetch)
           for (int half = 0; half < 2; ++half) {
             const uint32_t sh_addr = s_addr + half * 64;
             const uint32_t g = o_cnt + (uint32_t)(2 * j + half);  // half-units of this stream before this one
