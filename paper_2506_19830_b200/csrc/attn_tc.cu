@@ -793,9 +793,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant_
               tmem_ld64(o_addr + hf * 64, o);
               tc_wait_ld();
               if (ri.q_index >= 0) {
-                uint4 *dst = reinterpret_cast<uint4 *>(tc.partial_o + prow * kD + hf * 64);
+                // chunk-major: 16-byte chunk k of row r at [slot][k][r], so a warp's store is 512 contiguous bytes
+                uint4 *dst = reinterpret_cast<uint4 *>(tc.partial_o) + ((int64_t)slot * 32 + hf * 16) * 128 + r;
 #pragma unroll
-                for (int jj = 0; jj < 16; ++jj) dst[jj] = make_uint4(o[4 * jj], o[4 * jj + 1], o[4 * jj + 2], o[4 * jj + 3]);
+                for (int jj = 0; jj < 16; ++jj) dst[jj * 128] = make_uint4(o[4 * jj], o[4 * jj + 1], o[4 * jj + 2], o[4 * jj + 3]);
               }
             }
             if (ri.q_index >= 0) *reinterpret_cast<float2 *>(tc.partial_ml + prow * 2) = make_float2(m_used, l);
@@ -816,69 +817,55 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant_
 }
 
 // Merge of the partials of one M-tile: O = sum_j 2^(m_j - M) O_j / sum_j 2^(m_j - M) l_j.
-// One warp per query row (grid: targets x 16 CTAs of 8 warps); the slots are read in a fixed order.
+// One thread per (query row, 16-byte chunk of channels); a warp holds 32 consecutive rows of one chunk, which
+// is how the partials are laid out ([slot][chunk][row]).  Grid: targets x 16 CTAs of 256 threads.  The slots
+// are combined in a fixed order.
 __global__ void __launch_bounds__(256)
 attn_tc_merge_kernel(DevBatch d, DevTcPlan tc, uint16_t *__restrict__ out, float *__restrict__ lse) {
   const TcTarget g = tc.targets[blockIdx.x];
   const TcReq rq = tc.reqs[g.req];
   const int T = tc.tokens_per_mtile, G = d.group;
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int r = blockIdx.y * 8 + warp;
+  const int item = blockIdx.y * 256 + threadIdx.x;  // 0 .. 4095
+  const int k = item >> 7, r = item & 127;           // chunk of 4 channels, row
   const int tok = g.mtile * T + r / G;
   const bool live = r < T * G && tok < rq.n_q;
   // the partials come from the kernel launched just before this one
   asm volatile("griddepcontrol.wait;" ::: "memory");
   if (!live) return;
   const int64_t qi = (int64_t)(rq.q_row0 + tok) * d.n_q_heads + g.kv_head * G + r % G;
-  const int64_t prow0 = (int64_t)g.slot_begin * 128 + r;
-  float M = -INFINITY, L = 0.f;
+  const float2 *ml = reinterpret_cast<const float2 *>(tc.partial_ml) + (int64_t)g.slot_begin * 128 + r;
+  const float4 *po = reinterpret_cast<const float4 *>(tc.partial_o) + ((int64_t)g.slot_begin * 32 + k) * 128 + r;
+  float M = -INFINITY;
+  for (int j = 0; j < g.n_slots; ++j) {
+    const float2 v = ml[(int64_t)j * 128];
+    if (v.y > 0.f) M = fmaxf(M, v.x);  // a stream that saw no key of the row contributes nothing
+  }
+  float L = 0.f;
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-  for (int j0 = 0; j0 < g.n_slots; j0 += 32) {
-    // lane j holds (m, l) of slot j0 + j
-    const int j = j0 + lane;
-    float mj = -INFINITY, lj = 0.f;
-    if (j < g.n_slots) {
-      const float2 ml = *reinterpret_cast<const float2 *>(tc.partial_ml + (prow0 + (int64_t)j * 128) * 2);
-      if (ml.y > 0.f) {  // a stream that saw no key of the row contributes nothing
-        mj = ml.x;
-        lj = ml.y;
+  for (int j0 = 0; j0 < g.n_slots; j0 += 8) {
+    float4 o[8];
+    float2 v[8];
+#pragma unroll
+    for (int jj = 0; jj < 8; ++jj)
+      if (j0 + jj < g.n_slots) {
+        o[jj] = po[(int64_t)(j0 + jj) * 32 * 128];
+        v[jj] = ml[(int64_t)(j0 + jj) * 128];
       }
-    }
-    float mc = mj;
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) mc = fmaxf(mc, __shfl_xor_sync(0xFFFFFFFFu, mc, o));
-    const float M_new = fmaxf(M, mc);
-    if (M_new == -INFINITY) continue;
-    const float carry = (M == -INFINITY) ? 0.f : exp2f(M - M_new);
-    acc.x *= carry; acc.y *= carry; acc.z *= carry; acc.w *= carry;
-    L *= carry;
-    M = M_new;
-    const float w = (lj > 0.f) ? exp2f(mj - M) : 0.f;
-    const float wl = w * lj;
-    const int n = min(32, g.n_slots - j0);
-    for (int jb = 0; jb < n; jb += 8) {
-      float4 o[8];
-#pragma unroll
-      for (int k = 0; k < 8; ++k)
-        if (jb + k < n) o[k] = *reinterpret_cast<const float4 *>(tc.partial_o + (prow0 + (int64_t)(j0 + jb + k) * 128) * kD + lane * 4);
-#pragma unroll
-      for (int k = 0; k < 8; ++k)
-        if (jb + k < n) {
-          const float wj = __shfl_sync(0xFFFFFFFFu, w, jb + k);
-          L += __shfl_sync(0xFFFFFFFFu, wl, jb + k);
-          if (wj != 0.f) {
-            acc.x = fmaf(wj, o[k].x, acc.x);
-            acc.y = fmaf(wj, o[k].y, acc.y);
-            acc.z = fmaf(wj, o[k].z, acc.z);
-            acc.w = fmaf(wj, o[k].w, acc.w);
-          }
-        }
-    }
+    for (int jj = 0; jj < 8; ++jj)
+      if (j0 + jj < g.n_slots && v[jj].y > 0.f) {
+        const float w = exp2f(v[jj].x - M);
+        L = fmaf(w, v[jj].y, L);
+        acc.x = fmaf(w, o[jj].x, acc.x);
+        acc.y = fmaf(w, o[jj].y, acc.y);
+        acc.z = fmaf(w, o[jj].z, acc.z);
+        acc.w = fmaf(w, o[jj].w, acc.w);
+      }
   }
   const float inv = 1.0f / L;
   uint2 pk = make_uint2(pack_bf16(acc.x * inv, acc.y * inv), pack_bf16(acc.z * inv, acc.w * inv));
-  *reinterpret_cast<uint2 *>(out + qi * kD + lane * 4) = pk;
-  if (lse != nullptr && lane == 0) lse[qi] = (M + log2f(L)) * 0.6931471805599453f;
+  *reinterpret_cast<uint2 *>(out + qi * kD + k * 4) = pk;
+  if (lse != nullptr && k == 0) lse[qi] = (M + log2f(L)) * 0.6931471805599453f;
 }
 
 // ---- tensor maps -------------------------------------------------------------------

@@ -86,7 +86,7 @@ struct DevTcPlan {
   const TcTarget *targets;
   int32_t n_cta, n_targets;
   int32_t tokens_per_mtile;  // floor(128 / group)
-  float *partial_o;          // [n_slots][128][head_dim] fp32, unnormalised
+  float *partial_o;          // [n_slots][32 chunks of 4 channels][128 rows][4] fp32, unnormalised
   float *partial_ml;         // [n_slots][128][2] (reference exponent in log2 units, sum)
 };
 
