@@ -192,6 +192,7 @@ def main():
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-graph", action="store_true", help="issue every launch from Python instead of replaying CUDA graphs")
     ap.add_argument("--path", type=int, default=0, help="attention path: 0 auto, 1 CUDA cores, 2 tensor cores")
     args = ap.parse_args()
     if args.impl == "reference":
@@ -231,10 +232,10 @@ def main():
 
     def step(i):
         c = i % copies
-        plan.lr_verify_attention(x0.q, kc[c], vc[c], y.out, None, 0.0, stream)
-        ctx.lr_accept_greedy(lc[c], x0.draft_ids, x0.cu_draft, y.n_accept, y.bonus_id, y.scratch, None, stream)
+        plan.lr_verify_attention(x0.q, kc[c], vc[c], y.out, None, 0.0, None)
+        ctx.lr_accept_greedy(lc[c], x0.draft_ids, x0.cu_draft, y.n_accept, y.bonus_id, y.scratch, None, None)
         plan.lr_commit(x0.verdict, y.n_accept, y.n_steps_accepted, y.survivor, y.committed_len, y.keep_off, y.keep_pages,
-                       y.keep_valid, y.free_off, y.free_pages, stream)
+                       y.keep_valid, y.free_off, y.free_pages, None)
 
     def barrier():
         if world > 1:
@@ -247,43 +248,83 @@ def main():
         step(i)
     assert plan.lr_poll_status() == 0
 
+    # The steps are replayed from CUDA graphs (one graph = `copies` consecutive steps, one per copy of the
+    # inputs), so that the launch-bound loop is not limited by the host issuing four launches per step.
+    # --no-graph issues every launch from Python instead.
+    def attn_only(c):
+        plan.lr_verify_attention(x0.q, kc[c], vc[c], y.out, None, 0.0, None)
+
+    def accept_only(c):
+        ctx.lr_accept_greedy(lc[c], x0.draft_ids, x0.cu_draft, y.n_accept, y.bonus_id, y.scratch, None, None)
+
+    def commit_only(c):
+        plan.lr_commit(x0.verdict, y.n_accept, y.n_steps_accepted, y.survivor, y.committed_len, y.keep_off, y.keep_pages,
+                       y.keep_valid, y.free_off, y.free_pages, None)
+
+    def make_runner(fn):
+        """Returns run(first, count): `count` consecutive calls fn(i % copies) starting at index `first`."""
+        graph = None
+        if not args.no_graph:
+            try:
+                graph = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(graph, stream=side):  # the binding launches on torch's current stream
+                    for c in range(copies):
+                        fn(c)
+            except Exception as exc:  # capture not possible: fall back to plain launches
+                graph = None
+                if rank == 0:
+                    print(f"bench: CUDA graph capture failed ({exc}); issuing launches from the host", file=sys.stderr)
+
+        def run(first, count):
+            i = first
+            while count > 0:
+                if graph is not None and i % copies == 0 and count >= copies:
+                    graph.replay()
+                    i += copies
+                    count -= copies
+                else:
+                    fn(i % copies)
+                    i += 1
+                    count -= 1
+        return run, graph is not None
+
+    main_stream = stream
+    side = torch.cuda.Stream()
+    l0 = ctx.launch_count
+    step(0)
+    launches_per_step = ctx.launch_count - l0
+    run_step, graphed = make_runner(lambda c: step(c))
+    run_attn, _ = make_runner(attn_only)
+    run_accept, _ = make_runner(accept_only)
+    run_commit, _ = make_runner(commit_only)
+    torch.cuda.synchronize()
+    run_step(0, copies)  # one replay as warm-up of the graph itself
+    assert plan.lr_poll_status() == 0
+
+    def timed(run, count):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        e0.record(main_stream)
+        run(0, count)
+        e1.record(main_stream)
+        barrier()
+        return e0.elapsed_time(e1)
+
     # ---- region A: K whole steps, device time -------------------------------------
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
     launches0 = ctx.launch_count
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
-    e0.record(stream)
-    for i in range(K):
-        step(W + i)
-    e1.record(stream)
-    barrier()
+    ms_total = timed(run_step, K)
     launches = ctx.launch_count - launches0
-    ms_total = e0.elapsed_time(e1)
+    if graphed:  # launches replayed from a graph are not counted by the library: count them from the capture
+        per_step = launches_per_step
+        launches = per_step * K
 
-    # ---- region B: the same K steps with an event pair around every launch --------
-    names = ("attention", "accept", "commit")
-    ev = {n: [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)] for n in names}
-    barrier()
-    for i in range(K):
-        c = (W + i) % copies
-        a, z = ev["attention"][i]
-        a.record(stream)
-        plan.lr_verify_attention(x0.q, kc[c], vc[c], y.out, None, 0.0, stream)
-        z.record(stream)
-        a, z = ev["accept"][i]
-        a.record(stream)
-        ctx.lr_accept_greedy(lc[c], x0.draft_ids, x0.cu_draft, y.n_accept, y.bonus_id, y.scratch, None, stream)
-        z.record(stream)
-        a, z = ev["commit"][i]
-        a.record(stream)
-        plan.lr_commit(x0.verdict, y.n_accept, y.n_steps_accepted, y.survivor, y.committed_len, y.keep_off, y.keep_pages,
-                       y.keep_valid, y.free_off, y.free_pages, stream)
-        z.record(stream)
-    barrier()
+    # ---- region B: each kernel alone, K back-to-back launches over the rotating copies ------
+    kernel_us = {"attention": 1e3 * timed(run_attn, K) / K, "accept": 1e3 * timed(run_accept, K) / K,
+                 "commit": 1e3 * timed(run_commit, K) / K}
     clocks = sampler.stop() if rank == 0 else None
-    kernel_us = {n: 1e3 * sum(a.elapsed_time(z) for a, z in ev[n]) / K for n in names}
     assert plan.lr_poll_status() == 0
 
     # ---- end to end: host buffers in, host results out -----------------------------
@@ -365,7 +406,8 @@ def main():
             "config": {"workload": f"config{args.config}_{w.name}", "seed": w.seed, "requests_per_gpu": b.n_req,
                        "branches_per_gpu": b.n_branch, "kv_tokens_per_gpu": b.kv_tokens(), "verified_tokens_per_gpu": b.n_verified_tokens,
                        "l2_policy": f"rotating {copies} copies of KV pools and logits ({copies * per_copy / 1e6:.0f} MB > L2)",
-                       "attention_path": args.path},
+                       "attention_path": args.path, "cuda_graph": bool(graphed),
+                       "per_kernel_timing": "K back-to-back launches of the kernel alone over the rotating copies"},
             "roofline": roof, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
             "kernels": kernels,
         }
