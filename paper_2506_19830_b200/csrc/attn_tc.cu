@@ -423,7 +423,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant_
   asm volatile("griddepcontrol.wait;" ::: "memory");
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
-  const int piece0 = tc.cta_piece_off[blockIdx.x], piece1 = tc.cta_piece_off[blockIdx.x + 1];
+  const TcCtaHead *head = tc.heads + blockIdx.x;
+  const int piece0 = head->piece0, piece1 = head->piece1;
   const int T = tc.tokens_per_mtile;
   const int G = d.group;
 
@@ -438,8 +439,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant_
     bool ok = true;
     const uint32_t q_box_bytes = (uint32_t)(64 * G * T * 2);
     for (int pc = piece0; pc < piece1 && ok; ++pc) {
-      const TcPiece pi = tc.pieces[pc];
-      const TcReq rq = tc.reqs[pi.req];
+      const TcPiece pi = pc == piece0 ? head->first : tc.pieces[pc];
+      const TcReq rq = pc == piece0 ? head->first_req : tc.reqs[pi.req];
       const int n = pi.tile_end - pi.tile_begin;
       // Q tiles of the piece, once the MMAs of the previous piece no longer read the buffers
       ok = wait_bar(&ctrl->q_empty, (q_count & 1u) ^ 1u, ctrl, d.status, 205);
@@ -467,7 +468,17 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant_
         return pg;
       };
       int c_cur = pi.tile_begin >> 2;
-      int32_t pg_cur = load_chunk(c_cur), pg_nxt = load_chunk(c_cur + 1);
+      int32_t pg_nxt = load_chunk(c_cur + 1), pg_cur;
+      if (pc == piece0) {  // the first chunk of the first piece comes with the CTA head
+        pg_cur = head->first_pages[lane];
+        if (pg_cur >= d.n_pool_pages) {
+          d.status[0] = kDevBounds;
+          d.status[1] = 201;
+          pg_cur = 0;
+        }
+      } else {
+        pg_cur = load_chunk(c_cur);
+      }
       for (int i = 0; i < 2 * n && ok; ++i, ++ring) {
         bool is_v;
         const int t = pi.tile_begin + ord.step(i, is_v);
@@ -530,8 +541,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant_
         mma_ts(o_tmem, s_tmem + half * 64 + k4 * 8, b + (uint64_t)(k4 * (2048 >> 4)), kIdescPV, acc || k4 != 0);
     };
     for (int pc = piece0; pc < piece1 && ok; ++pc, ++pc_idx) {
-      const TcPiece pi = tc.pieces[pc];
-      const TcReq rq = tc.reqs[pi.req];
+      const TcPiece pi = pc == piece0 ? head->first : tc.pieces[pc];
+      const TcReq rq = pc == piece0 ? head->first_req : tc.reqs[pi.req];
       const int n = pi.tile_end - pi.tile_begin, mode = pi.n_mt;
       const RingOrder ord(n, mode);
       const int my_units = mode == 2 ? n : (n - s + 1) / 2;
@@ -650,8 +661,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant_
     uint32_t s_cnt = 0, o_cnt = 0;  // tiles / half-units of this stream so far
     bool ok = true;
     for (int pc = piece0; pc < piece1; ++pc) {
-      const TcPiece pi = tc.pieces[pc];
-      const TcReq rq = tc.reqs[pi.req];
+      const TcPiece pi = pc == piece0 ? head->first : tc.pieces[pc];
+      const TcReq rq = pc == piece0 ? head->first_req : tc.reqs[pi.req];
       const int n = pi.tile_end - pi.tile_begin, mode = pi.n_mt;
       const int my_units = mode == 2 ? n : (n - s + 1) / 2;
       if (ok && my_units > 0) {
@@ -823,16 +834,15 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant_
 __global__ void __launch_bounds__(256)
 attn_tc_merge_kernel(DevBatch d, DevTcPlan tc, uint16_t *__restrict__ out, float *__restrict__ lse) {
   const TcTarget g = tc.targets[blockIdx.x];
-  const TcReq rq = tc.reqs[g.req];
   const int T = tc.tokens_per_mtile, G = d.group;
   const int item = blockIdx.y * 256 + threadIdx.x;  // 0 .. 4095
   const int k = item >> 7, r = item & 127;           // chunk of 4 channels, row
   const int tok = g.mtile * T + r / G;
-  const bool live = r < T * G && tok < rq.n_q;
+  const bool live = r < T * G && tok < g.n_q;
   // the partials come from the kernel launched just before this one
   asm volatile("griddepcontrol.wait;" ::: "memory");
   if (!live) return;
-  const int64_t qi = (int64_t)(rq.q_row0 + tok) * d.n_q_heads + g.kv_head * G + r % G;
+  const int64_t qi = (int64_t)(g.q_row0 + tok) * d.n_q_heads + g.kv_head * G + r % G;
   const float2 *ml = reinterpret_cast<const float2 *>(tc.partial_ml) + (int64_t)g.slot_begin * 128 + r;
   const float4 *po = reinterpret_cast<const float4 *>(tc.partial_o) + ((int64_t)g.slot_begin * 32 + k) * 128 + r;
   float M = -INFINITY;
@@ -1054,6 +1064,7 @@ int tc_build_host_plan(const lr_ctx *ctx, const lr_batch *b, const int32_t *req_
       memset(&tg, 0, sizeof(tg));
       tg.req = g.req; tg.kv_head = g.kv; tg.mtile = g.mtile0 + mt;
       tg.slot_begin = n_slots; tg.n_slots = (int)contrib.size();
+      tg.q_row0 = reqs[g.req].q_row0; tg.n_q = reqs[g.req].n_q;
       for (int32_t *c : contrib) *c = n_slots++;
       targets.push_back(tg);
     }
@@ -1063,6 +1074,24 @@ int tc_build_host_plan(const lr_ctx *ctx, const lr_batch *b, const int32_t *req_
   out.n_targets = (int)targets.size();
   out.n_partial_slots = n_slots;
   out.tokens_per_mtile = T;
+  static_assert(sizeof(TcCtaHead) == 256, "one CTA head = 256 bytes");
+  std::vector<TcCtaHead> heads((size_t)n_cta);
+  for (int c = 0; c < n_cta; ++c) {
+    TcCtaHead &h = heads[c];
+    memset(&h, 0, sizeof(h));
+    h.piece0 = cta_off[c];
+    h.piece1 = cta_off[c + 1];
+    if (h.piece1 > h.piece0) {
+      h.first = pieces[h.piece0];
+      h.first_req = reqs[h.first.req];
+      const int c0 = h.first.tile_begin >> 2;
+      for (int k = 0; k < 32; ++k) {
+        const int idx = c0 * 32 + k;
+        h.first_pages[k] = idx < h.first_req.n_pages ? pages[(size_t)h.first_req.page_off + idx].page : -1;
+      }
+    }
+  }
+  out.o_heads = img.add(heads.data(), heads.size() * sizeof(TcCtaHead));
   out.o_pages = img.add(pages.data(), pages.size() * sizeof(TcPage));
   out.o_rows = img.add(rows.data(), rows.size() * sizeof(TcRow));
   out.o_pieces = img.add(pieces.data(), pieces.size() * sizeof(TcPiece));
@@ -1082,6 +1111,7 @@ void tc_bind_device_plan(const TcHostPlan &h, unsigned char *image_base, unsigne
   memset(&p->tc, 0, sizeof(p->tc));
   if (!h.ok) return;
   DevTcPlan &t = p->tc;
+  t.heads = reinterpret_cast<const TcCtaHead *>(image_base + h.o_heads);
   t.pages = reinterpret_cast<const TcPage *>(image_base + h.o_pages);
   t.rows = reinterpret_cast<const TcRow *>(image_base + h.o_rows);
   t.pieces = reinterpret_cast<const TcPiece *>(image_base + h.o_pieces);

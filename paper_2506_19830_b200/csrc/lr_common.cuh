@@ -75,9 +75,18 @@ struct TcReq {
 struct TcTarget {
   int32_t req, kv_head, mtile;
   int32_t slot_begin, n_slots;  // partial slots to merge (n_slots >= 2)
-  int32_t pad[3];
+  int32_t q_row0, n_q;          // query token range of the request (copied, to spare a dependent load)
+  int32_t pad;
+};
+struct TcCtaHead {    // everything a CTA needs to start, in one 256-byte record (one round trip to memory)
+  int32_t piece0, piece1;   // its pieces
+  TcPiece first;            // copy of pieces[piece0]
+  TcReq first_req;          // copy of reqs[first.req]
+  int32_t first_pages[32];  // physical ids of pages 32*c .. 32*c+31 of that request, c = first.tile_begin / 4; -1 = absent
+  int32_t pad[14];
 };
 struct DevTcPlan {
+  const TcCtaHead *heads;        // [n_cta]
   const TcPage *pages;
   const TcRow *rows;             // [n_q_rows]
   const TcPiece *pieces;
@@ -134,7 +143,7 @@ struct Image {
 // Host-side result of planning the tensor-core attention for one batch.
 struct TcHostPlan {
   bool ok = false;  // shape supported by the tensor-core path
-  size_t o_pages = 0, o_rows = 0, o_pieces = 0, o_cta_piece_off = 0, o_reqs = 0, o_targets = 0;  // image offsets
+  size_t o_heads = 0, o_pages = 0, o_rows = 0, o_pieces = 0, o_cta_piece_off = 0, o_reqs = 0, o_targets = 0;  // image offsets
   int n_cta = 0, n_targets = 0, n_pieces = 0, n_partial_slots = 0, tokens_per_mtile = 0;
   // scratch region behind the image: (exponent, sum) pairs, then fp32 partial outputs
   size_t s_ml = 0, s_o = 0, scratch_bytes = 0, scratch_zero_bytes = 0;
