@@ -188,17 +188,34 @@ accept_greedy_kernel(const uint16_t *__restrict__ logits, int64_t row_stride, in
   // ---- last CTA: per-branch longest matching prefix + bonus ------------------
   __threadfence();
   volatile unsigned long long *vk = row_key;
-  for (int b = tid; b < n_branch; b += kThreads) {
+  // One warp per branch: the L + 1 rows of a branch are loaded 32 at a time, all at once, and the first
+  // mismatch is found with a ballot -- no chain of dependent loads along the drafts.
+  const int lane = tid & 31;
+  for (int b = tid >> 5; b < n_branch; b += kThreads / 32) {
     const int32_t d0 = cu_draft[b], L = cu_draft[b + 1] - d0;
     const int32_t r0 = d0 + b;
-    int32_t n = 0;
-    while (n < L) {
-      int32_t t = (int32_t)(0xFFFFFFFFu - (uint32_t)(vk[r0 + n] & 0xFFFFFFFFull));
-      if (draft_ids[d0 + n] != t) break;
-      ++n;
+    int32_t n = L, bonus = 0;
+    bool found = false;
+    for (int32_t i0 = 0; i0 <= L && !found; i0 += 32) {
+      const int32_t i = i0 + lane;
+      int32_t t = 0;
+      bool mismatch = false;
+      if (i <= L) {
+        t = (int32_t)(0xFFFFFFFFu - (uint32_t)(vk[r0 + i] & 0xFFFFFFFFull));
+        mismatch = (i == L) || (draft_ids[d0 + i] != t);  // row L has no draft: the scan always stops there
+      }
+      const unsigned m = __ballot_sync(0xFFFFFFFFu, mismatch);
+      if (m != 0u) {
+        const int first = __ffs(m) - 1;
+        n = i0 + first;
+        bonus = __shfl_sync(0xFFFFFFFFu, t, first);
+        found = true;
+      }
     }
-    n_accept[b] = n;
-    bonus_id[b] = (int32_t)(0xFFFFFFFFu - (uint32_t)(vk[r0 + n] & 0xFFFFFFFFull));
+    if (lane == 0) {
+      n_accept[b] = n;
+      bonus_id[b] = bonus;
+    }
   }
   if (row_argmax != nullptr)
     for (int r = tid; r < n_rows; r += kThreads)
