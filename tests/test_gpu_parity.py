@@ -111,6 +111,33 @@ def test_increasing_scores_force_running_max_updates():
     check_attention(y.out, y.lse, o_ref, l_ref)
 
 
+def test_score_jumps_force_the_exact_redo_of_a_half_unit():
+    """A few late keys score ~70 nats above everything before them (more than 2^64 in the kernel's log2
+    units): the sweep that runs against the stale reference exponent must notice and redo the half-unit
+    with its own maximum.  One jump sits in the prefix, one in a segment, one in a branch tail."""
+    rng = _rng(11)
+    model = Model(8, 2, 128, 64)
+    batch = build_batch(model, [{"P": 1100, "segs": [40, 24], "branches": [(1, 20, 16, 16), (2, 9, 9, 9)]}], rng)
+    k, v = fill_kv(batch, rng, poison="nan")
+    q = bf16_round(np.ones((batch.n_q_rows, 8, 128), dtype=np.float32))
+    kf = bf16_round(np.zeros(k.shape, dtype=np.float32))
+    big = np.float32(70.0 * np.sqrt(128) / 128)  # q . k * scale = 70
+    spans = [(int(batch.span_slot[0]), 700), (int(batch.span_slot[0]), 1000), (int(batch.span_slot[1]), 17),
+             (int(batch.br_own_slot[0]), 3), (int(batch.br_own_slot[1]), 8)]
+    for n, (slot, tok) in enumerate(spans):
+        pg = batch.page_ids[slot + tok // 16]
+        kf[pg, :, tok % 16, :] = bf16_round(np.full((2, 128), big * (1 + 0.5 * n), dtype=np.float32))
+    kf[k == 0x7FC0] = 0x7FC0  # keep the poison where the generator put it
+    ctx = B.Context(model, 0)
+    plan = B.Plan(ctx, batch)
+    x = R.DeviceInputs(batch, type("T", (), dict(q=q, k_pool=kf, v_pool=v, logits=None, draft_ids=None, verdict=None)), with_logits=False)
+    y = R.PassOutputs(batch)
+    plan.lr_verify_attention(x.q, x.k_pool, x.v_pool, y.out, y.lse)
+    assert plan.lr_poll_status() == 0
+    o_ref, l_ref = O.verify_attention(batch, q, kf, v)
+    check_attention(y.out, y.lse, o_ref, l_ref)
+
+
 def test_accept_special_rows_and_ties():
     """Natural ties, ties across vector / chunk boundaries, -0/+0, NaN, inf, and a vocab that is not a multiple of 8."""
     rng = _rng(5)
