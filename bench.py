@@ -204,6 +204,7 @@ def main():
     from lr_workloads import make_config
     from paper_2506_19830_b200 import binding as B
     from paper_2506_19830_b200 import runner as R
+    from paper_2506_19830_b200 import sharding as S
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -215,7 +216,7 @@ def main():
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device(dev))
 
-    w = make_config(args.config, seed=20250619 + args.config + 1000 * rank)
+    w = make_config(args.config, seed=S.rank_seed(20250619 + args.config, rank))
     b, t = w.batch, w.tensors
     ctx = B.Context(b.model, local)
     plan = B.Plan(ctx, b)
@@ -355,22 +356,16 @@ def main():
             plan.lr_verify_pass_host(io, kc[(W + i) % copies], vc[(W + i) % copies], staging, 0.0, stream)
         torch.cuda.synchronize()
         e2e_s = (time.perf_counter() - t0) / Ke
-        e2e_t = torch.tensor([e2e_s], device=dev, dtype=torch.float64)
-        if world > 1:
-            dist.all_reduce(e2e_t, op=dist.ReduceOp.MAX)
-        e2e = {"value": world * b.n_verified_tokens / float(e2e_t.item()), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
-               "d2h_bytes_per_step": int(d2h), "ms_per_step": float(e2e_t.item()) * 1e3, "steps": Ke,
+        e2e_ms, e2e_tokens = S.reduce_measurement(e2e_s * 1e3, b.n_verified_tokens, dev)
+        e2e = {"value": S.job_throughput(e2e_ms, e2e_tokens), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
+               "d2h_bytes_per_step": int(d2h), "ms_per_step": e2e_ms, "steps": Ke,
                "note": "lr_verify_pass_host: pinned host Q/logits/drafts/verdicts in, all results out, stream sync per step; "
                        "KV pools are device-resident cache state"}
 
     # ---- aggregate over ranks --------------------------------------------------------
-    tmax = torch.tensor([ms_total], device=dev, dtype=torch.float64)
-    tok = torch.tensor([float(b.n_verified_tokens)], device=dev, dtype=torch.float64)
-    if world > 1:
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        dist.all_reduce(tok, op=dist.ReduceOp.SUM)
-    ms_step = float(tmax.item()) / K
-    value = float(tok.item()) / (ms_step * 1e-3)
+    ms_max, tokens_total = S.reduce_measurement(ms_total, b.n_verified_tokens, dev)
+    ms_step = ms_max / K
+    value = S.job_throughput(ms_step, tokens_total)
 
     if rank == 0:
         hbm_peak, tc_peak, peak_kind = _peaks()
