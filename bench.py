@@ -192,6 +192,7 @@ def main():
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-overlap", action="store_true", help="run the three steps of a pass strictly one after another")
     ap.add_argument("--no-graph", action="store_true", help="issue every launch from Python instead of replaying CUDA graphs")
     ap.add_argument("--path", type=int, default=0, help="attention path: 0 auto, 1 CUDA cores, 2 tensor cores")
     args = ap.parse_args()
@@ -231,8 +232,13 @@ def main():
     lc = [x0.logits] + [x0.logits.clone() for _ in range(copies - 1)]
     stream = torch.cuda.current_stream()
 
+    overlap_stream = None if args.no_overlap else torch.cuda.Stream()
+
     def step(i):
         c = i % copies
+        if overlap_stream is not None:  # attention || (acceptance -> commit): the two chains share no data
+            R.run_pass_overlapped(ctx, plan, x0, y, overlap_stream, kc[c], vc[c], lc[c])
+            return
         plan.lr_verify_attention(x0.q, kc[c], vc[c], y.out, None, 0.0, None)
         ctx.lr_accept_greedy(lc[c], x0.draft_ids, x0.cu_draft, y.n_accept, y.bonus_id, y.scratch, None, None)
         plan.lr_commit(x0.verdict, y.n_accept, y.n_steps_accepted, y.survivor, y.committed_len, y.keep_off, y.keep_pages,
@@ -401,7 +407,7 @@ def main():
             "config": {"workload": f"config{args.config}_{w.name}", "seed": w.seed, "requests_per_gpu": b.n_req,
                        "branches_per_gpu": b.n_branch, "kv_tokens_per_gpu": b.kv_tokens(), "verified_tokens_per_gpu": b.n_verified_tokens,
                        "l2_policy": f"rotating {copies} copies of KV pools and logits ({copies * per_copy / 1e6:.0f} MB > L2)",
-                       "attention_path": args.path, "cuda_graph": bool(graphed),
+                       "attention_path": args.path, "cuda_graph": bool(graphed), "overlap": "attention || (accept -> commit) on two streams" if overlap_stream is not None else "none",
                        "per_kernel_timing": "K back-to-back launches of the kernel alone over the rotating copies"},
             "roofline": roof, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
             "kernels": kernels,

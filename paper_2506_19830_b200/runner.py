@@ -82,3 +82,25 @@ def run_pass(ctx: B.Context, plan: B.Plan, x: DeviceInputs, y: PassOutputs, stre
                          y.row_argmax if want_row_argmax else None, stream)
     plan.lr_commit(x.verdict, y.n_accept, y.n_steps_accepted, y.survivor, y.committed_len, y.keep_off, y.keep_pages,
                    y.keep_valid, y.free_off, y.free_pages, stream)
+
+
+def run_pass_overlapped(ctx: B.Context, plan: B.Plan, x: DeviceInputs, y: PassOutputs, side: torch.cuda.Stream,
+                        k_pool=None, v_pool=None, logits=None):
+    """One whole verify pass with the two independent chains on two streams: attention on the current
+    stream, acceptance -> commit (which need nothing from attention) on ``side``; both are joined back
+    into the current stream.  Works under CUDA-graph capture (fork/join through events)."""
+    main = torch.cuda.current_stream()
+    k_pool = x.k_pool if k_pool is None else k_pool
+    v_pool = x.v_pool if v_pool is None else v_pool
+    logits = x.logits if logits is None else logits
+    fork = torch.cuda.Event()
+    fork.record(main)
+    side.wait_event(fork)
+    with torch.cuda.stream(side):
+        ctx.lr_accept_greedy(logits, x.draft_ids, x.cu_draft, y.n_accept, y.bonus_id, y.scratch, None, None)
+        plan.lr_commit(x.verdict, y.n_accept, y.n_steps_accepted, y.survivor, y.committed_len, y.keep_off, y.keep_pages,
+                       y.keep_valid, y.free_off, y.free_pages, None)
+        join = torch.cuda.Event()
+        join.record(side)
+    plan.lr_verify_attention(x.q, k_pool, v_pool, y.out, None, 0.0, None)
+    main.wait_event(join)

@@ -41,6 +41,26 @@ def test_whole_pass_ragged_small(seed):
     run_and_check_pass(make_random_small(1000 + seed))
 
 
+def test_overlapped_pass_gives_the_same_results():
+    """Attention on one stream, acceptance -> commit on another (they share no data): same outputs."""
+    w = make_config(2)
+    b, t = w.batch, w.tensors
+    ctx = B.Context(b.model, 0)
+    plan = B.Plan(ctx, b)
+    x = R.DeviceInputs(b, t)
+    y = R.PassOutputs(b)
+    side = torch.cuda.Stream()
+    for _ in range(3):
+        R.run_pass_overlapped(ctx, plan, x, y, side)
+    torch.cuda.synchronize()
+    assert plan.lr_poll_status() == 0
+    o_ref, _ = O.verify_attention(b, t.q, t.k_pool, t.v_pool)
+    check_attention(y.out, None, o_ref, None)
+    n_ref, bonus_ref, _ = O.accept_greedy(t.logits, t.draft_ids, b.cu_draft)
+    assert np.array_equal(y.n_accept.cpu().numpy(), n_ref) and np.array_equal(y.bonus_id.cpu().numpy(), bonus_ref)
+    check_commit(y.commit_dict(), O.commit(b, t.verdict, n_ref))
+
+
 @pytest.mark.parametrize("cfg", [1, 2])
 def test_generic_attention_path(cfg):
     run_and_check_pass(make_config(cfg), path=B.PATH_GENERIC)
