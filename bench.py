@@ -383,8 +383,11 @@ def main():
         else:
             roof = {"bound": "tensor", "achieved": a_flops / t_att / 1e12, "peak": tc_peak, "unit": "TFLOP/s"}
         roof["frac"] = roof["achieved"] / roof["peak"]
-        roof.update({"traffic": None, "kernel": "lr_verify_attention", "kernel_us": kernel_us["attention"],
-                     "algorithmic_bytes": a_bytes, "algorithmic_flops": a_flops, "peak_source": f"of {peak_kind}",
+        # dram__bytes_read.sum + dram__bytes_write.sum of one attn_tc_kernel launch on this workload (ncu
+        # captures summarised under profiles/, taken on the kernels as they are); None where not captured
+        traffic = {2: 17_960_704 + 0, 3: 274_865_152 + 8_119_808}.get(args.config) if args.path == 0 else None
+        roof.update({"traffic": traffic, "kernel": "lr_verify_attention", "kernel_us": kernel_us["attention"],
+                     "algorithmic_bytes": a_bytes, "algorithmic_flops": a_flops, "peak_source": f"of {peak_kind}", "timed": "attn_tc_kernel + attn_tc_merge_kernel",
                      "roofline_us": max(hbm_time, tc_time) * 1e6})
         acc_b = accept_bytes(b)
         kernels = {
