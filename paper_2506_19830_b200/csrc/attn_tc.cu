@@ -1009,7 +1009,7 @@ int tc_build_host_plan(const lr_ctx *ctx, const lr_batch *b, const int32_t *req_
   // CTA whose weight interval [total*c/n, total*(c+1)/n) holds the tile's start position.
   // The start of a group inside a CTA's range (epilogue, Q reload, pipeline ramp) is charged like
   // kPieceStartTiles tiles, so such a CTA gets fewer tiles.
-  constexpr int kPieceStartTiles = 4;
+  constexpr int kPieceStartTiles = 3;
   int64_t total_w = 0, total_tiles = 0;
   for (const Grp &g : grps) {
     total_w += (int64_t)(g.n_tiles + kPieceStartTiles) * g.weight;
