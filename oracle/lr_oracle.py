@@ -22,6 +22,10 @@ What is computed, and where the paper fixes it:
   taken from the target distribution at that position.  Greedy reading: a draft
   is accepted iff it equals the argmax of the target logits (lowest index on
   ties); the extra ("bonus") token is the argmax of the row where it halted.
+* ``accept_sample``     -- the same passage read literally: rejection sampling with acceptance
+  probability min(1, P/Q) and a final token from the residual distribution, for point-mass draft
+  distributions (prompt-lookup drafts, the paper's SD method), temperature sampling, random numbers
+  passed in.
 * ``commit``            -- Algorithm 1, last two lines: j* = min({j : V(s_j, s^_j)
   = False} U {gamma}); output = s^_0 .. s^_{j*-1} (+) s_{j*}.  On the KV cache
   this keeps the prefix pages, the pages of the first j* segments and the pages
@@ -32,7 +36,9 @@ Pins (tests/test_oracle_*.py): textbook decode attention, torch SDPA causal
 attention on each branch's concatenated sequence, closed forms that expose the
 visibility sets, brute force over explicit token lists, LSE merge identity,
 page-permutation / poison invariance; acceptance against pure-Python scans,
-all 2^L match patterns and the (1-a^{L+1})/(1-a) mean; commit against an
+all 2^L match patterns and the (1-a^{L+1})/(1-a) mean; stochastic acceptance against the
+exactness theorem of speculative sampling (output distribution = target distribution, by
+integrating over the uniforms), a hand-computed example, its greedy limit and scipy's softmax; commit against an
 independent token-level list model and the closed-form E[j*].
 """
 from __future__ import annotations
@@ -238,6 +244,64 @@ def commit(batch, verdict: np.ndarray, n_accept: np.ndarray):
         "free_off": i32(free_off),
         "free_pages": i32(free_pages),
     }
+
+
+# ---------------------------------------------------------------------------
+# a2'. stochastic token-level acceptance (rejection sampling)
+# ---------------------------------------------------------------------------
+def target_probs(logits_row_bits: np.ndarray, temperature: float) -> np.ndarray:
+    """P = softmax(logits / T) of one row, float64 (NaN logits count as -inf)."""
+    x = bf16_bits_to_f64(logits_row_bits) / float(temperature)
+    x = np.where(np.isnan(x), -np.inf, x)
+    w = np.exp(x - x.max())
+    return w / w.sum()
+
+
+def sample_inverse_cdf(weights: np.ndarray, u: float) -> int:
+    """Smallest index v with cumsum(weights)[v] > u * sum(weights)  (u in [0, 1))."""
+    c = np.cumsum(weights)
+    return int(np.searchsorted(c, u * c[-1], side="right"))
+
+
+def accept_sample(logits_bits: np.ndarray, draft_ids: np.ndarray, cu_draft: np.ndarray, temperature: float,
+                  u_accept: np.ndarray, u_final: np.ndarray):
+    """Rejection sampling of Background, "Speculative Decoding", for drafts whose draft distribution Q
+    is a point mass at the drafted token (prompt-lookup / n-gram drafts, the paper's SD method):
+
+    drafts are processed in order; draft i is accepted with probability min(1, P_i(d_i) / Q_i(d_i)) =
+    P_i(d_i), here iff u_accept[i] < P_i(d_i); at the first rejection the process halts and the final
+    token is sampled from the normalised max(0, P_i - Q_i), i.e. P_i with the rejected token removed;
+    if every draft is accepted the final token is sampled from P of the extra row.  Sampling is by
+    inverse CDF with u_final[b].  A draft id outside the vocabulary has probability 0.
+    Returns (n_accept, final_id, p_draft) with p_draft[i] = P_i(d_i).
+    """
+    V = logits_bits.shape[1]
+    B = len(cu_draft) - 1
+    n_accept = np.zeros(B, dtype=np.int32)
+    final_id = np.zeros(B, dtype=np.int32)
+    p_draft = np.zeros(int(cu_draft[-1]), dtype=np.float64)
+    for b in range(B):
+        d0, L = int(cu_draft[b]), int(cu_draft[b + 1] - cu_draft[b])
+        row0 = d0 + b
+        n = 0
+        residual = None
+        while n < L:
+            P = target_probs(logits_bits[row0 + n], temperature)
+            d = int(draft_ids[d0 + n])
+            pd = P[d] if 0 <= d < V else 0.0
+            p_draft[d0 + n] = pd
+            if float(u_accept[d0 + n]) < pd:
+                n += 1  # accepted; next draft
+                continue
+            residual = P.copy()  # rejected: halt, resample from P with the rejected token removed
+            if 0 <= d < V:
+                residual[d] = 0.0
+            break
+        if residual is None:  # all accepted: one more token from the target
+            residual = target_probs(logits_bits[row0 + L], temperature)
+        n_accept[b] = n
+        final_id[b] = sample_inverse_cdf(residual, float(u_final[b]))
+    return n_accept, final_id, p_draft
 
 
 def verify_pass(batch, q_bits, k_pool_bits, v_pool_bits, logits_bits, draft_ids, verdict):
