@@ -177,6 +177,33 @@ int lr_accept_greedy(lr_ctx *ctx, const void *logits_d, int64_t row_stride_elems
                      void *scratch_d, void *stream);
 
 /*
+ * Stochastic token-level acceptance (Background, "Speculative Decoding": a
+ * rejection-sampling procedure processes the proposed tokens in order; an
+ * accepted token is kept, at the first rejection the process halts and a final
+ * token is sampled from the target's distribution), for drafts whose draft
+ * distribution is a point mass at the drafted token (prompt-lookup / n-gram
+ * drafts, the paper's SD method).  With P_i = softmax(logits[row0_b + i] / T):
+ *     draft i is accepted iff u_accept[cu_draft[b] + i] < P_i(d_i)   (= min(1, P/Q));
+ *     n_b     = number of drafts accepted before the first rejection;
+ *     final_b = inverse-CDF sample with u_final[b] (smallest v whose cumulative
+ *               weight exceeds u * total) from P_{n_b} with the rejected token
+ *               removed, or from P_{L_b} when every draft was accepted.
+ * The uniforms (in [0, 1)) are inputs: the call draws no random numbers.  A draft
+ * id outside [0, vocab) has probability 0.  Arithmetic is fp32; a decision whose
+ * uniform lies within rounding of its threshold may differ from an exact
+ * evaluation.  p_draft_d (nullable, [sum L_b]) receives P_i(d_i) for the drafts
+ * up to and including the first rejected one.  Rows, strides and alignment as
+ * for lr_accept_greedy; temperature must be > 0; at most 65535 rows per call.
+ * scratch_d: lr_accept_sample_scratch_bytes bytes, 8-byte aligned, no initial
+ * contents needed; calls sharing it must not overlap on the device.
+ */
+int lr_accept_sample_scratch_bytes(const lr_ctx *ctx, int32_t n_rows, size_t *bytes_out);
+int lr_accept_sample(lr_ctx *ctx, const void *logits_d, int64_t row_stride_elems, const int32_t *draft_ids_d,
+                     const int32_t *cu_draft_d, int32_t n_branch, int32_t n_rows, float temperature,
+                     const float *u_accept_d, const float *u_final_d, int32_t *n_accept_d, int32_t *final_id_d,
+                     float *p_draft_d, void *scratch_d, void *stream);
+
+/*
  * lr_accept_greedy without a caller-provided scratch buffer.  (The paper has no
  * counterpart: this is a packaging variant of the call above, same results.)
  *

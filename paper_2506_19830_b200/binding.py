@@ -76,6 +76,8 @@ def lib() -> C.CDLL:
             "lr_accept_scratch_bytes": [i32, C.POINTER(sz)],
             "lr_accept_greedy": [vp, vp, i64, vp, vp, i32, i32, vp, vp, vp, vp, vp],
             "lr_accept_greedy_static": [vp, vp, i64, vp, vp, i32, i32, vp, vp, vp, vp],
+            "lr_accept_sample_scratch_bytes": [vp, i32, C.POINTER(sz)],
+            "lr_accept_sample": [vp, vp, i64, vp, vp, i32, i32, f32, vp, vp, vp, vp, vp, vp, vp],
             "lr_commit": [vp] + [vp] * 10 + [vp],
             "lr_pass_staging_bytes": [vp, C.POINTER(sz)],
             "lr_verify_pass_host": [vp, C.POINTER(lr_pass_host_io), vp, vp, vp, sz, f32, vp],
@@ -187,6 +189,20 @@ class Context:
         _check(lib().lr_accept_greedy_static(self.handle, _ptr(logits), logits.stride(0), _ptr(draft_ids), _ptr(cu_draft),
                                              n_branch, logits.shape[0], _ptr(n_accept), _ptr(bonus_id), _ptr(row_argmax),
                                              _stream_ptr(stream)), "lr_accept_greedy_static")
+
+    def lr_accept_sample(self, logits: torch.Tensor, draft_ids: torch.Tensor, cu_draft: torch.Tensor, temperature: float,
+                         u_accept: torch.Tensor, u_final: torch.Tensor, n_accept: torch.Tensor, final_id: torch.Tensor,
+                         scratch: torch.Tensor, p_draft: Optional[torch.Tensor] = None, stream=None) -> None:
+        """Rejection-sampling acceptance; u_accept [sum L] and u_final [n_branch] are fp32 uniforms in [0, 1)."""
+        n_branch = cu_draft.numel() - 1
+        _check(lib().lr_accept_sample(self.handle, _ptr(logits), logits.stride(0), _ptr(draft_ids), _ptr(cu_draft), n_branch,
+                                      logits.shape[0], float(temperature), _ptr(u_accept), _ptr(u_final), _ptr(n_accept),
+                                      _ptr(final_id), _ptr(p_draft), _ptr(scratch), _stream_ptr(stream)), "lr_accept_sample")
+
+    def accept_sample_scratch(self, n_rows: int) -> torch.Tensor:
+        n = C.c_size_t()
+        _check(lib().lr_accept_sample_scratch_bytes(self.handle, n_rows, C.byref(n)), "lr_accept_sample_scratch_bytes")
+        return torch.empty((n.value + 7) // 8, dtype=torch.int64, device=f"cuda:{self.device}")
 
     @staticmethod
     def accept_scratch(n_rows: int, device) -> torch.Tensor:

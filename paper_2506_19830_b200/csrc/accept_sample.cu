@@ -1,0 +1,293 @@
+// Stochastic token-level acceptance (rejection sampling) for point-mass draft distributions.
+//
+// Two kernels.  accept_stats_kernel streams the bf16 logits once -- the HBM-bound part: grid (chunks of 8192
+// logits, rows); a CTA reduces its chunk to (raw maximum M_c, S_c = sum exp((x - M_c) / T)) and stores the pair.
+// accept_sample_kernel, one CTA per branch, combines the pairs of a row in chunk order into (m, Z), gets
+// P_i(d_i) = exp((x_d - m) / T) / Z for the drafts, walks the acceptance chain u_i < P_i(d_i), and draws the
+// final token by inverse CDF over the stop row with the rejected token removed: first over the chunk
+// weights S_c exp((M_c - m) / T) (no second pass over the row), then inside the one chunk that holds the
+// target, which is read again and prefix-summed.  Every reduction has a fixed order: same inputs, same output.
+#include <algorithm>
+
+#include "lr_common.cuh"
+
+namespace lr {
+
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kVec = 4;                       // 16-byte vectors per thread
+constexpr int kChunk = kThreads * kVec * 8;   // logits per chunk
+constexpr int kRowBatch = 32;                 // rows of a branch handled at a time in the chain
+
+__device__ __forceinline__ uint4 ld_stream(const uint4 *p) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+  return v;
+}
+__device__ __forceinline__ float bf_lo(uint32_t u) { return __uint_as_float(u << 16); }
+__device__ __forceinline__ float bf_hi(uint32_t u) { return __uint_as_float(u & 0xFFFF0000u); }
+__device__ __forceinline__ float denan(float x) { return (x != x) ? -INFINITY : x; }  // NaN counts as -inf
+
+// the 32 logits of thread `tid` in chunk `c` of a row: element e = c*kChunk + (k*kThreads + tid)*8 + j for the
+// striped layout (coalesced), or e = c*kChunk + tid*32 + k*8 + j for the blocked layout (contiguous per thread)
+template <bool kBlocked>
+__device__ __forceinline__ void load_chunk(const uint16_t *rp, int32_t vocab, int c, int tid, float (&x)[kVec * 8]) {
+  const int32_t n_vec = vocab >> 3;
+#pragma unroll
+  for (int k = 0; k < kVec; ++k) {
+    const int32_t vi = c * (kChunk / 8) + (kBlocked ? tid * kVec + k : k * kThreads + tid);
+    if (vi < n_vec) {
+      const uint4 v = ld_stream(reinterpret_cast<const uint4 *>(rp) + vi);
+      const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        x[k * 8 + 2 * j] = denan(bf_lo(w[j]));
+        x[k * 8 + 2 * j + 1] = denan(bf_hi(w[j]));
+      }
+    } else {
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {  // ragged end of the row (vocab not a multiple of 8), or beyond it
+        const int32_t e = vi * 8 + j;
+        x[k * 8 + j] = e < vocab ? denan(bf_lo((uint32_t)rp[e])) : -INFINITY;
+      }
+    }
+  }
+}
+
+__device__ __forceinline__ float block_reduce_max(float v, float *s_red) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xFFFFFFFFu, v, o));
+  if ((threadIdx.x & 31) == 0) s_red[threadIdx.x >> 5] = v;
+  __syncthreads();
+  float r = s_red[0];
+#pragma unroll
+  for (int w = 1; w < kThreads / 32; ++w) r = fmaxf(r, s_red[w]);
+  __syncthreads();
+  return r;
+}
+__device__ __forceinline__ float block_reduce_sum(float v, float *s_red) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+  if ((threadIdx.x & 31) == 0) s_red[threadIdx.x >> 5] = v;
+  __syncthreads();
+  float r = s_red[0];
+#pragma unroll
+  for (int w = 1; w < kThreads / 32; ++w) r += s_red[w];
+  __syncthreads();
+  return r;
+}
+
+__global__ void __launch_bounds__(kThreads)
+accept_stats_kernel(const uint16_t *__restrict__ logits, int64_t row_stride, int32_t vocab, float k_log2,
+                    float2 *__restrict__ stats) {
+  __shared__ float s_red[kThreads / 32];
+  const int c = blockIdx.x, row = blockIdx.y, n_chunks = gridDim.x;
+  asm volatile("griddepcontrol.wait;" ::: "memory");  // the logits may come from the kernel launched just before
+  float x[kVec * 8];
+  load_chunk<false>(logits + (int64_t)row * row_stride, vocab, c, threadIdx.x, x);
+  float m = -INFINITY;
+#pragma unroll
+  for (int i = 0; i < kVec * 8; ++i) m = fmaxf(m, x[i]);
+  const float M = block_reduce_max(m, s_red);
+  float sum = 0.f;
+  if (M > -INFINITY) {
+    const float off = -M * k_log2;
+#pragma unroll
+    for (int i = 0; i < kVec * 8; ++i) sum += exp2f(fmaf(x[i], k_log2, off));
+  }
+  const float S = block_reduce_sum(sum, s_red);
+  if (threadIdx.x == 0) stats[(int64_t)row * n_chunks + c] = make_float2(M, S);
+}
+
+__global__ void __launch_bounds__(kThreads)
+accept_sample_kernel(const uint16_t *__restrict__ logits, int64_t row_stride, int32_t vocab, float k_log2,
+                     const float2 *__restrict__ stats, int n_chunks, const int32_t *__restrict__ draft_ids,
+                     const int32_t *__restrict__ cu_draft, const float *__restrict__ u_accept,
+                     const float *__restrict__ u_final, int32_t *__restrict__ n_accept, int32_t *__restrict__ final_id,
+                     float *__restrict__ p_draft) {
+  __shared__ float s_red[kThreads / 32];
+  __shared__ float s_m[kRowBatch], s_p[kRowBatch];
+  __shared__ int s_n, s_stop;
+  __shared__ float s_stop_m;
+  __shared__ int s_pick_chunk, s_pick_thread;
+  __shared__ float s_pick_before;
+  const int b = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  asm volatile("griddepcontrol.wait;" ::: "memory");  // the statistics come from the kernel launched just before
+  const int32_t d0 = cu_draft[b], L = cu_draft[b + 1] - d0, r0 = d0 + b;
+
+  // ---- acceptance chain, kRowBatch rows at a time: one warp per row combines the row's chunk pairs in order
+  if (tid == 0) {
+    s_n = L;
+    s_stop = 0;
+  }
+  __syncthreads();
+  for (int i0 = 0; i0 <= L; i0 += kRowBatch) {
+    for (int i = i0 + warp; i < min(i0 + kRowBatch, L + 1); i += kThreads / 32) {
+      const float2 *st = stats + (int64_t)(r0 + i) * n_chunks;
+      float m = -INFINITY;
+      for (int c = lane; c < n_chunks; c += 32) m = fmaxf(m, st[c].x);
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
+      float z = 0.f;
+      for (int c0 = 0; c0 < n_chunks; c0 += 32) {  // chunk order: 32 at a time, butterfly inside
+        const int c = c0 + lane;
+        float t = 0.f;
+        if (c < n_chunks) {
+          const float2 v = st[c];
+          if (v.y > 0.f) t = v.y * exp2f((v.x - m) * k_log2);
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xFFFFFFFFu, t, o);
+        z += t;
+      }
+      if (lane == 0) {
+        float p = 0.f;
+        if (i < L) {
+          const int32_t dtok = draft_ids[d0 + i];
+          if (dtok >= 0 && dtok < vocab && z > 0.f) {
+            const float xd = denan(bf_lo((uint32_t)logits[(int64_t)(r0 + i) * row_stride + dtok]));
+            p = exp2f((xd - m) * k_log2) / z;
+          }
+          if (p_draft != nullptr) p_draft[d0 + i] = p;
+        }
+        s_m[i - i0] = m;
+        s_p[i - i0] = p;
+      }
+    }
+    __syncthreads();
+    if (tid == 0 && !s_stop) {
+      for (int i = i0; i < min(i0 + kRowBatch, L + 1); ++i) {
+        if (i == L || !(u_accept[d0 + i] < s_p[i - i0])) {  // rejected (or no draft left): halt here
+          s_n = i;
+          s_stop = 1;
+          s_stop_m = s_m[i - i0];
+          break;
+        }
+      }
+    }
+    __syncthreads();
+    if (s_stop) break;
+  }
+  const int n = s_n;
+  const float m = s_stop_m;
+  const int64_t stop_row = r0 + n;
+  const uint16_t *rp = logits + stop_row * row_stride;
+  const int32_t dead = n < L ? draft_ids[d0 + n] : -1;  // the rejected token has weight 0 in the residual
+  float w_dead = 0.f;
+  if (dead >= 0 && dead < vocab) w_dead = exp2f((denan(bf_lo((uint32_t)rp[dead])) - m) * k_log2);
+
+  // ---- which chunk holds the target: sequential over the chunk weights (a few dozen)
+  if (tid == 0) {
+    const float2 *st = stats + stop_row * n_chunks;
+    const int dead_chunk = (dead >= 0 && dead < vocab) ? dead / kChunk : -1;
+    float total = 0.f;
+    for (int c = 0; c < n_chunks; ++c) {
+      const float2 v = st[c];
+      float w = v.y > 0.f ? v.y * exp2f((v.x - m) * k_log2) : 0.f;
+      if (c == dead_chunk) w = fmaxf(w - w_dead, 0.f);
+      total += w;
+    }
+    const float target = u_final[b] * total;
+    float cum = 0.f;
+    int pick = -1, last_nonzero = 0;
+    for (int c = 0; c < n_chunks; ++c) {
+      const float2 v = st[c];
+      float w = v.y > 0.f ? v.y * exp2f((v.x - m) * k_log2) : 0.f;
+      if (c == dead_chunk) w = fmaxf(w - w_dead, 0.f);
+      if (w > 0.f) last_nonzero = c;
+      if (cum + w > target) {
+        pick = c;
+        break;
+      }
+      cum += w;
+    }
+    if (pick < 0) {  // rounding pushed the target past the last chunk: take the last chunk with any weight
+      pick = last_nonzero;
+      cum = target;
+    }
+    s_pick_chunk = pick;
+    s_pick_before = target - cum;  // what is still to be covered inside the chunk
+  }
+  __syncthreads();
+
+  // ---- inside the chunk: thread t owns 32 consecutive logits; exclusive scan of the thread sums, then a
+  //      sequential walk in the one thread whose range holds the target
+  const int pc = s_pick_chunk;
+  const float remain = s_pick_before;
+  float x[kVec * 8];
+  load_chunk<true>(rp, vocab, pc, tid, x);
+  float w[kVec * 8], mine = 0.f;
+#pragma unroll
+  for (int i = 0; i < kVec * 8; ++i) {
+    const int32_t e = pc * kChunk + tid * 32 + i;
+    w[i] = (e == dead || x[i] == -INFINITY) ? 0.f : exp2f((x[i] - m) * k_log2);
+    mine += w[i];
+  }
+  float incl = mine;  // inclusive scan over the block, in thread order
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const float y = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+    if (lane >= o) incl += y;
+  }
+  if (lane == 31) s_red[warp] = incl;
+  if (tid == 0) s_pick_thread = -1;
+  __syncthreads();
+  float base = 0.f;
+  for (int k = 0; k < warp; ++k) base += s_red[k];
+  const float before = base + incl - mine;
+  const bool holds = before <= remain && before + mine > remain && mine > 0.f;
+  if (holds) atomicMax(&s_pick_thread, tid);  // rounding can make two neighbours claim it: the later one decides
+  __syncthreads();
+  int pt = s_pick_thread;
+  if (pt < 0) {  // rounding pushed the target past the end of the chunk: the last thread with any weight
+    if (mine > 0.f) atomicMax(&s_pick_thread, tid);
+    __syncthreads();
+    pt = s_pick_thread;
+  }
+  if (tid == max(pt, 0)) {
+    float cum = before;
+    int pick = -1, last = 0;
+#pragma unroll
+    for (int i = 0; i < kVec * 8; ++i) {
+      if (w[i] > 0.f) {
+        last = i;
+        if (pick < 0 && cum + w[i] > remain) pick = i;
+        cum += w[i];
+      }
+    }
+    if (pick < 0) pick = last;
+    n_accept[b] = n;
+    final_id[b] = pc * kChunk + tid * 32 + pick;
+  }
+}
+
+}  // namespace
+
+size_t accept_sample_scratch_bytes(int32_t vocab, int32_t n_rows) {
+  const size_t n_chunks = ((size_t)vocab + kChunk - 1) / kChunk;
+  return std::max<size_t>(8, (size_t)n_rows * n_chunks * sizeof(float2));
+}
+
+int launch_accept_sample(lr_ctx *ctx, const void *logits, int64_t stride, const int32_t *drafts, const int32_t *cu_draft,
+                         int32_t n_branch, int32_t n_rows, float temperature, const float *u_accept, const float *u_final,
+                         int32_t *n_accept, int32_t *final_id, float *p_draft, void *scratch, cudaStream_t s) {
+  const int32_t vocab = ctx->model.vocab;
+  const int n_chunks = (vocab + kChunk - 1) / kChunk;
+  if (n_rows > 65535) {
+    set_error("lr_accept_sample: more than 65535 logits rows in one call");
+    return LR_EUNSUPPORTED;
+  }
+  const float k_log2 = 1.4426950408889634f / temperature;
+  auto *lg = reinterpret_cast<const uint16_t *>(logits);
+  auto *st = reinterpret_cast<float2 *>(scratch);
+  accept_stats_kernel<<<dim3((unsigned)n_chunks, (unsigned)n_rows), kThreads, 0, s>>>(lg, stride, vocab, k_log2, st);
+  ctx->launches++;
+  if (int rc = cuda_fail(cudaGetLastError(), "accept_stats_kernel launch")) return rc;
+  accept_sample_kernel<<<(unsigned)n_branch, kThreads, 0, s>>>(lg, stride, vocab, k_log2, st, n_chunks, drafts, cu_draft, u_accept,
+                                                              u_final, n_accept, final_id, p_draft);
+  ctx->launches++;
+  return cuda_fail(cudaGetLastError(), "accept_sample_kernel launch");
+}
+
+}  // namespace lr

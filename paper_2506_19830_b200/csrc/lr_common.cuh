@@ -168,6 +168,10 @@ int launch_accept(lr_ctx *ctx, const void *logits, int64_t stride, const int32_t
 int launch_accept_static(lr_ctx *ctx, const void *logits, int64_t stride, const int32_t *drafts, const int32_t *cu_draft,
                          int32_t n_branch, int32_t n_rows, int32_t *n_accept, int32_t *bonus, int32_t *row_argmax,
                          cudaStream_t s);
+size_t accept_sample_scratch_bytes(int32_t vocab, int32_t n_rows);
+int launch_accept_sample(lr_ctx *ctx, const void *logits, int64_t stride, const int32_t *drafts, const int32_t *cu_draft,
+                         int32_t n_branch, int32_t n_rows, float temperature, const float *u_accept, const float *u_final,
+                         int32_t *n_accept, int32_t *final_id, float *p_draft, void *scratch, cudaStream_t s);
 int launch_commit(lr_plan *p, const uint8_t *verdict, const int32_t *n_accept, int32_t *n_steps, int32_t *survivor,
                   int32_t *committed, int32_t *keep_off, int32_t *keep_pages, int32_t *keep_valid, int32_t *free_off,
                   int32_t *free_pages, cudaStream_t s);
