@@ -268,6 +268,17 @@ def main():
         plan.lr_commit(x0.verdict, y.n_accept, y.n_steps_accepted, y.survivor, y.committed_len, y.keep_off, y.keep_pages,
                        y.keep_valid, y.free_off, y.free_pages, None)
 
+    # the stochastic acceptance rule (not part of the timed step: the step uses the greedy rule), timed alone
+    rs = np.random.default_rng(w.seed)
+    u_acc = torch.from_numpy(rs.uniform(0, 1, max(1, len(t.draft_ids))).astype(np.float32)).to(dev)
+    u_fin = torch.from_numpy(rs.uniform(0, 1, b.n_branch).astype(np.float32)).to(dev)
+    samp_scratch = ctx.accept_sample_scratch(b.n_logit_rows)
+    samp_n = torch.empty(b.n_branch, dtype=torch.int32, device=dev)
+    samp_f = torch.empty(b.n_branch, dtype=torch.int32, device=dev)
+
+    def sample_only(c):
+        ctx.lr_accept_sample(lc[c], x0.draft_ids, x0.cu_draft, 0.6, u_acc, u_fin, samp_n, samp_f, samp_scratch, None, None)
+
     def make_runner(fn):
         """Returns run(first, count): `count` consecutive calls fn(i % copies) starting at index `first`."""
         graph = None
@@ -304,6 +315,7 @@ def main():
     run_attn, _ = make_runner(attn_only)
     run_accept, _ = make_runner(accept_only)
     run_commit, _ = make_runner(commit_only)
+    run_sample, _ = make_runner(sample_only)
     torch.cuda.synchronize()
     run_step(0, copies)  # one replay as warm-up of the graph itself
     assert plan.lr_poll_status() == 0
@@ -330,7 +342,7 @@ def main():
 
     # ---- region B: each kernel alone, K back-to-back launches over the rotating copies ------
     kernel_us = {"attention": 1e3 * timed(run_attn, K) / K, "accept": 1e3 * timed(run_accept, K) / K,
-                 "commit": 1e3 * timed(run_commit, K) / K}
+                 "commit": 1e3 * timed(run_commit, K) / K, "sample": 1e3 * timed(run_sample, K) / K}
     clocks = sampler.stop() if rank == 0 else None
     assert plan.lr_poll_status() == 0
 
@@ -397,6 +409,10 @@ def main():
                                  "frac_of_hbm_peak": acc_b / (kernel_us["accept"] * 1e-6) / 1e9 / hbm_peak,
                                  "algorithmic_bytes": acc_b},
             "lr_commit": {"us": kernel_us["commit"]},
+            "lr_accept_sample": {"us": kernel_us["sample"], "GB/s": acc_b / (kernel_us["sample"] * 1e-6) / 1e9,
+                                 "frac_of_hbm_peak": acc_b / (kernel_us["sample"] * 1e-6) / 1e9 / hbm_peak,
+                                 "algorithmic_bytes": acc_b, "temperature": 0.6,
+                                 "note": "rejection-sampling acceptance; not part of the timed step"},
         }
         cpu = None
         if not args.no_cpu_baseline:

@@ -27,6 +27,11 @@ __device__ __forceinline__ uint4 ld_stream(const uint4 *p) {
 }
 __device__ __forceinline__ float bf_lo(uint32_t u) { return __uint_as_float(u << 16); }
 __device__ __forceinline__ float bf_hi(uint32_t u) { return __uint_as_float(u & 0xFFFF0000u); }
+__device__ __forceinline__ float ex2_approx(float x) {  // one MUFU operation; -inf gives 0
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
 __device__ __forceinline__ float denan(float x) { return (x != x) ? -INFINITY : x; }  // NaN counts as -inf
 
 // the 32 logits of thread `tid` in chunk `c` of a row: element e = c*kChunk + (k*kThreads + tid)*8 + j for the
@@ -93,8 +98,15 @@ accept_stats_kernel(const uint16_t *__restrict__ logits, int64_t row_stride, int
   float sum = 0.f;
   if (M > -INFINITY) {
     const float off = -M * k_log2;
+    float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;  // independent chains
 #pragma unroll
-    for (int i = 0; i < kVec * 8; ++i) sum += exp2f(fmaf(x[i], k_log2, off));
+    for (int i = 0; i < kVec * 8; i += 4) {
+      a0 += ex2_approx(fmaf(x[i], k_log2, off));
+      a1 += ex2_approx(fmaf(x[i + 1], k_log2, off));
+      a2 += ex2_approx(fmaf(x[i + 2], k_log2, off));
+      a3 += ex2_approx(fmaf(x[i + 3], k_log2, off));
+    }
+    sum = (a0 + a1) + (a2 + a3);
   }
   const float S = block_reduce_sum(sum, s_red);
   if (threadIdx.x == 0) stats[(int64_t)row * n_chunks + c] = make_float2(M, S);
@@ -106,25 +118,46 @@ accept_sample_kernel(const uint16_t *__restrict__ logits, int64_t row_stride, in
                      const int32_t *__restrict__ cu_draft, const float *__restrict__ u_accept,
                      const float *__restrict__ u_final, int32_t *__restrict__ n_accept, int32_t *__restrict__ final_id,
                      float *__restrict__ p_draft) {
+  extern __shared__ float2 s_st[];  // [kRowBatch][n_chunks]: the chunk pairs of a batch of rows
   __shared__ float s_red[kThreads / 32];
-  __shared__ float s_m[kRowBatch], s_p[kRowBatch];
+  __shared__ float s_m[kRowBatch], s_p[kRowBatch], s_u[kRowBatch], s_xd[kRowBatch];
+  __shared__ int32_t s_tok[kRowBatch];
   __shared__ int s_n, s_stop;
-  __shared__ float s_stop_m;
   __shared__ int s_pick_chunk, s_pick_thread;
   __shared__ float s_pick_before;
   const int b = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   asm volatile("griddepcontrol.wait;" ::: "memory");  // the statistics come from the kernel launched just before
   const int32_t d0 = cu_draft[b], L = cu_draft[b + 1] - d0, r0 = d0 + b;
 
-  // ---- acceptance chain, kRowBatch rows at a time: one warp per row combines the row's chunk pairs in order
+  // ---- acceptance chain, kRowBatch rows at a time.  Everything a batch needs from global memory (the chunk
+  //      pairs of its rows, the drafts, their logits, their uniforms) is fetched at once into shared memory.
   if (tid == 0) {
     s_n = L;
     s_stop = 0;
   }
-  __syncthreads();
-  for (int i0 = 0; i0 <= L; i0 += kRowBatch) {
-    for (int i = i0 + warp; i < min(i0 + kRowBatch, L + 1); i += kThreads / 32) {
-      const float2 *st = stats + (int64_t)(r0 + i) * n_chunks;
+  int i0 = 0;
+  for (;; i0 += kRowBatch) {
+    const int rows = min(kRowBatch, L + 1 - i0);
+    __syncthreads();
+    const float2 *src = stats + (int64_t)(r0 + i0) * n_chunks;  // consecutive rows are contiguous
+    for (int idx = tid; idx < rows * n_chunks; idx += kThreads) s_st[idx] = src[idx];
+    if (tid < rows) {
+      const int i = i0 + tid;
+      int32_t dtok = -1;
+      float xd = -INFINITY, u = 2.f;  // row L has no draft: u = 2 never passes
+      if (i < L) {
+        dtok = draft_ids[d0 + i];
+        u = u_accept[d0 + i];
+        if (dtok >= 0 && dtok < vocab) xd = denan(bf_lo((uint32_t)logits[(int64_t)(r0 + i) * row_stride + dtok]));
+        else dtok = -1;
+      }
+      s_tok[tid] = dtok;
+      s_xd[tid] = xd;
+      s_u[tid] = u;
+    }
+    __syncthreads();
+    for (int k = warp; k < rows; k += kThreads / 32) {  // one warp per row combines the row's chunk pairs in order
+      const float2 *st = s_st + k * n_chunks;
       float m = -INFINITY;
       for (int c = lane; c < n_chunks; c += 32) m = fmaxf(m, st[c].x);
 #pragma unroll
@@ -142,45 +175,35 @@ accept_sample_kernel(const uint16_t *__restrict__ logits, int64_t row_stride, in
         z += t;
       }
       if (lane == 0) {
-        float p = 0.f;
-        if (i < L) {
-          const int32_t dtok = draft_ids[d0 + i];
-          if (dtok >= 0 && dtok < vocab && z > 0.f) {
-            const float xd = denan(bf_lo((uint32_t)logits[(int64_t)(r0 + i) * row_stride + dtok]));
-            p = exp2f((xd - m) * k_log2) / z;
-          }
-          if (p_draft != nullptr) p_draft[d0 + i] = p;
-        }
-        s_m[i - i0] = m;
-        s_p[i - i0] = p;
+        const float p = (s_tok[k] >= 0 && z > 0.f) ? exp2f((s_xd[k] - m) * k_log2) / z : 0.f;
+        if (p_draft != nullptr && i0 + k < L) p_draft[d0 + i0 + k] = p;
+        s_m[k] = m;
+        s_p[k] = p;
       }
     }
     __syncthreads();
-    if (tid == 0 && !s_stop) {
-      for (int i = i0; i < min(i0 + kRowBatch, L + 1); ++i) {
-        if (i == L || !(u_accept[d0 + i] < s_p[i - i0])) {  // rejected (or no draft left): halt here
-          s_n = i;
+    if (tid == 0) {
+      for (int k = 0; k < rows; ++k)
+        if (!(s_u[k] < s_p[k])) {  // rejected (or no draft left): halt here
+          s_n = i0 + k;
           s_stop = 1;
-          s_stop_m = s_m[i - i0];
           break;
         }
-      }
     }
     __syncthreads();
     if (s_stop) break;
   }
-  const int n = s_n;
-  const float m = s_stop_m;
+  const int n = s_n, kn = n - i0;  // the stop row is row kn of the batch in shared memory
+  const float m = s_m[kn];
   const int64_t stop_row = r0 + n;
   const uint16_t *rp = logits + stop_row * row_stride;
-  const int32_t dead = n < L ? draft_ids[d0 + n] : -1;  // the rejected token has weight 0 in the residual
-  float w_dead = 0.f;
-  if (dead >= 0 && dead < vocab) w_dead = exp2f((denan(bf_lo((uint32_t)rp[dead])) - m) * k_log2);
+  const int32_t dead = n < L ? s_tok[kn] : -1;  // the rejected token has weight 0 in the residual
+  const float w_dead = dead >= 0 ? exp2f((s_xd[kn] - m) * k_log2) : 0.f;
 
-  // ---- which chunk holds the target: sequential over the chunk weights (a few dozen)
+  // ---- which chunk holds the target: sequential over the chunk weights (a few dozen, in shared memory)
   if (tid == 0) {
-    const float2 *st = stats + stop_row * n_chunks;
-    const int dead_chunk = (dead >= 0 && dead < vocab) ? dead / kChunk : -1;
+    const float2 *st = s_st + kn * n_chunks;
+    const int dead_chunk = dead >= 0 ? dead / kChunk : -1;
     float total = 0.f;
     for (int c = 0; c < n_chunks; ++c) {
       const float2 v = st[c];
@@ -284,7 +307,12 @@ int launch_accept_sample(lr_ctx *ctx, const void *logits, int64_t stride, const 
   accept_stats_kernel<<<dim3((unsigned)n_chunks, (unsigned)n_rows), kThreads, 0, s>>>(lg, stride, vocab, k_log2, st);
   ctx->launches++;
   if (int rc = cuda_fail(cudaGetLastError(), "accept_stats_kernel launch")) return rc;
-  accept_sample_kernel<<<(unsigned)n_branch, kThreads, 0, s>>>(lg, stride, vocab, k_log2, st, n_chunks, drafts, cu_draft, u_accept,
+  const size_t smem = (size_t)kRowBatch * n_chunks * sizeof(float2);
+  if (smem > 40 * 1024) {
+    set_error("lr_accept_sample: vocabulary of %d entries needs %zu bytes of shared memory per branch (limit 40 KB)", vocab, smem);
+    return LR_EUNSUPPORTED;
+  }
+  accept_sample_kernel<<<(unsigned)n_branch, kThreads, smem, s>>>(lg, stride, vocab, k_log2, st, n_chunks, drafts, cu_draft, u_accept,
                                                               u_final, n_accept, final_id, p_draft);
   ctx->launches++;
   return cuda_fail(cudaGetLastError(), "accept_sample_kernel launch");
