@@ -32,7 +32,7 @@ __device__ __forceinline__ float ex2_approx(float x) {  // one MUFU operation; -
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
-__device__ __forceinline__ float denan(float x) { return (x != x) ? -INFINITY : x; }  // NaN counts as -inf
+__device__ __forceinline__ float denan(float x) { return fmaxf(x, -INFINITY); }  // NaN counts as -inf (max drops a NaN operand)
 
 // the 32 logits of thread `tid` in chunk `c` of a row: element e = c*kChunk + (k*kThreads + tid)*8 + j for the
 // striped layout (coalesced), or e = c*kChunk + tid*32 + k*8 + j for the blocked layout (contiguous per thread)
@@ -91,14 +91,19 @@ accept_stats_kernel(const uint16_t *__restrict__ logits, int64_t row_stride, int
   asm volatile("griddepcontrol.wait;" ::: "memory");  // the logits may come from the kernel launched just before
   float x[kVec * 8];
   load_chunk<false>(logits + (int64_t)row * row_stride, vocab, c, threadIdx.x, x);
-  float m = -INFINITY;
+  float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;  // independent chains
 #pragma unroll
-  for (int i = 0; i < kVec * 8; ++i) m = fmaxf(m, x[i]);
-  const float M = block_reduce_max(m, s_red);
+  for (int i = 0; i < kVec * 8; i += 4) {
+    m0 = fmaxf(m0, x[i]);
+    m1 = fmaxf(m1, x[i + 1]);
+    m2 = fmaxf(m2, x[i + 2]);
+    m3 = fmaxf(m3, x[i + 3]);
+  }
+  const float M = block_reduce_max(fmaxf(fmaxf(m0, m1), fmaxf(m2, m3)), s_red);
   float sum = 0.f;
   if (M > -INFINITY) {
     const float off = -M * k_log2;
-    float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;  // independent chains
+    float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
 #pragma unroll
     for (int i = 0; i < kVec * 8; i += 4) {
       a0 += ex2_approx(fmaf(x[i], k_log2, off));
