@@ -89,6 +89,7 @@ accept_stats_kernel(const uint16_t *__restrict__ logits, int64_t row_stride, int
   __shared__ float s_red[kThreads / 32];
   const int c = blockIdx.x, row = blockIdx.y, n_chunks = gridDim.x;
   asm volatile("griddepcontrol.wait;" ::: "memory");  // the logits may come from the kernel launched just before
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   float x[kVec * 8];
   load_chunk<false>(logits + (int64_t)row * row_stride, vocab, c, threadIdx.x, x);
   float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;  // independent chains
@@ -133,6 +134,8 @@ accept_sample_kernel(const uint16_t *__restrict__ logits, int64_t row_stride, in
   const int b = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   asm volatile("griddepcontrol.wait;" ::: "memory");  // the statistics come from the kernel launched just before
   const int32_t d0 = cu_draft[b], L = cu_draft[b + 1] - d0, r0 = d0 + b;
+  const float u_fin = u_final[b];  // fetched early: needed only after the chain
+  static_assert(kRowBatch == 32, "the chain uses one lane per row of a batch");
 
   // ---- acceptance chain, kRowBatch rows at a time.  Everything a batch needs from global memory (the chunk
   //      pairs of its rows, the drafts, their logits, their uniforms) is fetched at once into shared memory.
@@ -187,13 +190,13 @@ accept_sample_kernel(const uint16_t *__restrict__ logits, int64_t row_stride, in
       }
     }
     __syncthreads();
-    if (tid == 0) {
-      for (int k = 0; k < rows; ++k)
-        if (!(s_u[k] < s_p[k])) {  // rejected (or no draft left): halt here
-          s_n = i0 + k;
-          s_stop = 1;
-          break;
-        }
+    if (warp == 0) {  // first rejected draft of the batch (kRowBatch == 32 rows = one per lane)
+      const bool rej = lane < rows && !(s_u[lane] < s_p[lane]);  // row L has no draft: always "rejected"
+      const unsigned mask = __ballot_sync(0xFFFFFFFFu, rej);
+      if (lane == 0 && mask != 0u) {
+        s_n = i0 + __ffs(mask) - 1;
+        s_stop = 1;
+      }
     }
     __syncthreads();
     if (s_stop) break;
@@ -205,37 +208,58 @@ accept_sample_kernel(const uint16_t *__restrict__ logits, int64_t row_stride, in
   const int32_t dead = n < L ? s_tok[kn] : -1;  // the rejected token has weight 0 in the residual
   const float w_dead = dead >= 0 ? exp2f((s_xd[kn] - m) * k_log2) : 0.f;
 
-  // ---- which chunk holds the target: sequential over the chunk weights (a few dozen, in shared memory)
-  if (tid == 0) {
+  // ---- which chunk holds the target: warp 0 scans the chunk weights, 32 chunks at a time (inclusive prefix
+  //      sums by shuffles, fixed order)
+  if (warp == 0) {
     const float2 *st = s_st + kn * n_chunks;
     const int dead_chunk = dead >= 0 ? dead / kChunk : -1;
+    auto weight = [&](int c) -> float {
+      if (c >= n_chunks) return 0.f;
+      const float2 v = st[c];
+      float w = v.y > 0.f ? v.y * exp2f((v.x - m) * k_log2) : 0.f;
+      if (c == dead_chunk) w = fmaxf(w - w_dead, 0.f);
+      return w;
+    };
     float total = 0.f;
-    for (int c = 0; c < n_chunks; ++c) {
-      const float2 v = st[c];
-      float w = v.y > 0.f ? v.y * exp2f((v.x - m) * k_log2) : 0.f;
-      if (c == dead_chunk) w = fmaxf(w - w_dead, 0.f);
-      total += w;
-    }
-    const float target = u_final[b] * total;
-    float cum = 0.f;
-    int pick = -1, last_nonzero = 0;
-    for (int c = 0; c < n_chunks; ++c) {
-      const float2 v = st[c];
-      float w = v.y > 0.f ? v.y * exp2f((v.x - m) * k_log2) : 0.f;
-      if (c == dead_chunk) w = fmaxf(w - w_dead, 0.f);
-      if (w > 0.f) last_nonzero = c;
-      if (cum + w > target) {
-        pick = c;
-        break;
+    for (int c0 = 0; c0 < n_chunks; c0 += 32) {
+      float t = weight(c0 + lane);
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const float y = __shfl_up_sync(0xFFFFFFFFu, t, o);
+        if (lane >= o) t += y;
       }
-      cum += w;
+      total += __shfl_sync(0xFFFFFFFFu, t, 31);
+    }
+    const float target = u_fin * total;
+    float base = 0.f;
+    int pick = -1, last_nonzero = 0;
+    float before = 0.f;
+    for (int c0 = 0; c0 < n_chunks && pick < 0; c0 += 32) {
+      const float w = weight(c0 + lane);
+      float t = w;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const float y = __shfl_up_sync(0xFFFFFFFFu, t, o);
+        if (lane >= o) t += y;
+      }
+      const unsigned nz = __ballot_sync(0xFFFFFFFFu, w > 0.f);
+      if (nz != 0u) last_nonzero = c0 + 31 - __clz(nz);
+      const unsigned hit = __ballot_sync(0xFFFFFFFFu, w > 0.f && base + t > target);
+      if (hit != 0u) {
+        const int l = __ffs(hit) - 1;
+        pick = c0 + l;
+        before = base + __shfl_sync(0xFFFFFFFFu, t - w, l);
+      }
+      base += __shfl_sync(0xFFFFFFFFu, t, 31);
     }
     if (pick < 0) {  // rounding pushed the target past the last chunk: take the last chunk with any weight
       pick = last_nonzero;
-      cum = target;
+      before = target;
     }
-    s_pick_chunk = pick;
-    s_pick_before = target - cum;  // what is still to be covered inside the chunk
+    if (lane == 0) {
+      s_pick_chunk = pick;
+      s_pick_before = target - before;  // what is still to be covered inside the chunk
+    }
   }
   __syncthreads();
 
@@ -317,10 +341,22 @@ int launch_accept_sample(lr_ctx *ctx, const void *logits, int64_t stride, const 
     set_error("lr_accept_sample: vocabulary of %d entries needs %zu bytes of shared memory per branch (limit 40 KB)", vocab, smem);
     return LR_EUNSUPPORTED;
   }
-  accept_sample_kernel<<<(unsigned)n_branch, kThreads, smem, s>>>(lg, stride, vocab, k_log2, st, n_chunks, drafts, cu_draft, u_accept,
-                                                              u_final, n_accept, final_id, p_draft);
+  // programmatic dependent launch: the per-branch grid is set up while the streaming grid drains
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof(cfg));
+  cfg.gridDim = dim3((unsigned)n_branch, 1, 1);
+  cfg.blockDim = dim3(kThreads, 1, 1);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  cudaError_t e = cudaLaunchKernelEx(&cfg, accept_sample_kernel, lg, stride, vocab, k_log2, (const float2 *)st, n_chunks, drafts,
+                                     cu_draft, u_accept, u_final, n_accept, final_id, p_draft);
   ctx->launches++;
-  return cuda_fail(cudaGetLastError(), "accept_sample_kernel launch");
+  return cuda_fail(e, "accept_sample_kernel launch");
 }
 
 }  // namespace lr
