@@ -154,7 +154,7 @@ def run_reference(args):
         return 0
     from lr_workloads import make_config
 
-    w = make_config(args.config)
+    w = make_config(args.config, carry_in=args.carry_in)
     tokens = w.batch.n_verified_tokens
     for _ in range(args.warmup):
         oracle_pass_seconds(w, 0.0, 1)
@@ -192,6 +192,7 @@ def main():
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--carry-in", action="store_true", help="q_len = L + 1 per branch (the last accepted token is a query too)")
     ap.add_argument("--no-overlap", action="store_true", help="run the three steps of a pass strictly one after another")
     ap.add_argument("--no-graph", action="store_true", help="issue every launch from Python instead of replaying CUDA graphs")
     ap.add_argument("--path", type=int, default=0, help="attention path: 0 auto, 1 CUDA cores, 2 tensor cores")
@@ -217,7 +218,7 @@ def main():
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device(dev))
 
-    w = make_config(args.config, seed=S.rank_seed(20250619 + args.config, rank))
+    w = make_config(args.config, seed=S.rank_seed(20250619 + args.config, rank), carry_in=args.carry_in)
     b, t = w.batch, w.tensors
     ctx = B.Context(b.model, local)
     plan = B.Plan(ctx, b)
@@ -397,7 +398,8 @@ def main():
         roof["frac"] = roof["achieved"] / roof["peak"]
         # dram__bytes_read.sum + dram__bytes_write.sum of one attn_tc_kernel launch on this workload (ncu
         # captures summarised under profiles/, taken on the kernels as they are); None where not captured
-        traffic = {2: 17_960_704 + 0, 3: 274_865_152 + 8_119_808}.get(args.config) if args.path == 0 else None
+        traffic = ({2: 17_960_704 + 0, 3: 274_865_152 + 8_119_808}.get(args.config)
+                   if args.path == 0 and not args.carry_in else None)
         roof.update({"traffic": traffic, "kernel": "lr_verify_attention", "kernel_us": kernel_us["attention"],
                      "algorithmic_bytes": a_bytes, "algorithmic_flops": a_flops, "peak_source": f"of {peak_kind}", "timed": "attn_tc_kernel + attn_tc_merge_kernel",
                      "roofline_us": max(hbm_time, tc_time) * 1e6})
@@ -426,7 +428,7 @@ def main():
             "config": {"workload": f"config{args.config}_{w.name}", "seed": w.seed, "requests_per_gpu": b.n_req,
                        "branches_per_gpu": b.n_branch, "kv_tokens_per_gpu": b.kv_tokens(), "verified_tokens_per_gpu": b.n_verified_tokens,
                        "l2_policy": f"rotating {copies} copies of KV pools and logits ({copies * per_copy / 1e6:.0f} MB > L2)",
-                       "attention_path": args.path, "cuda_graph": bool(graphed), "overlap": "attention || (accept -> commit) on two streams" if overlap_stream is not None else "none",
+                       "attention_path": args.path, "carry_in": bool(args.carry_in), "cuda_graph": bool(graphed), "overlap": "attention || (accept -> commit) on two streams" if overlap_stream is not None else "none",
                        "per_kernel_timing": "K back-to-back launches of the kernel alone over the rotating copies"},
             "roofline": roof, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
             "kernels": kernels,

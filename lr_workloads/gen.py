@@ -343,13 +343,16 @@ def fill_verdicts(batch: Batch, rng: np.random.Generator, p_accept: float) -> np
 # --------------------------------------------------------------------------
 # the five configurations
 # --------------------------------------------------------------------------
-def _chain_request(P: int, segs: Sequence[int], L: int) -> dict:
-    """Branch j (j = 1..gamma) sees segments 1..j; own_len = q_len = n_draft = L."""
-    return {"P": P, "segs": list(segs), "branches": [(j, L, L, L) for j in range(1, len(segs) + 1)]}
+def _chain_request(P: int, segs: Sequence[int], L: int, carry_in: bool = False) -> dict:
+    """Branch j (j = 1..gamma) sees segments 1..j; own_len = q_len = n_draft = L.  With ``carry_in`` the
+    tail also holds the last accepted token in front of the L drafts and it is a query too (own_len = q_len
+    = L + 1): the L + 1 query rows are then exactly the rows whose logits the acceptance step reads."""
+    q = L + 1 if carry_in else L
+    return {"P": P, "segs": list(segs), "branches": [(j, q, q, L) for j in range(1, len(segs) + 1)]}
 
 
 def make_config(idx: int, seed: Optional[int] = None, with_logits: bool = True, with_kv: bool = True,
-                poison: str = "nan") -> Workload:
+                poison: str = "nan", carry_in: bool = False) -> Workload:
     """Workload ``idx`` (1..5) of the benchmark suite; seed defaults to 20250619 + idx."""
     if seed is None:
         seed = 20250619 + idx
@@ -357,19 +360,19 @@ def make_config(idx: int, seed: Optional[int] = None, with_logits: bool = True, 
     k_scale = None
     if idx == 1:
         model = Model(4, 1, 64, 1024)
-        reqs = [_chain_request(256, [24, 24], 8)]
+        reqs = [_chain_request(256, [24, 24], 8, carry_in)]
         p_geo, p_ver = 0.3, 0.7
     elif idx == 2:
         model = Model(40, 8, 128, 152064)
-        reqs = [_chain_request(4096, [32] * 3, 16)]
+        reqs = [_chain_request(4096, [32] * 3, 16, carry_in)]
         p_geo, p_ver = 0.25, 0.6
     elif idx == 3:
         model = Model(40, 8, 128, 152064)
-        reqs = [_chain_request(16384, [48] * 4, 8) for _ in range(4)]
+        reqs = [_chain_request(16384, [48] * 4, 8, carry_in) for _ in range(4)]
         p_geo, p_ver = 0.25, 0.6
     elif idx == 4:
         model = Model(32, 8, 128, 152064)
-        reqs = [_chain_request(32768, [40] * 6, 16)]
+        reqs = [_chain_request(32768, [40] * 6, 16, carry_in)]
         p_geo, p_ver = 0.2, 0.6
     elif idx == 5:
         model = Model(40, 8, 128, 152064)
@@ -379,7 +382,7 @@ def make_config(idx: int, seed: Optional[int] = None, with_logits: bool = True, 
             gamma = int(rng.integers(2, 6 + 1))
             segs = [int(v) for v in rng.integers(16, 64 + 1, size=gamma)]
             L = int(rng.choice([4, 8, 16]))
-            reqs.append(_chain_request(P, segs, L))
+            reqs.append(_chain_request(P, segs, L, carry_in))
         p_geo, p_ver = 0.25, 0.6
     else:
         raise ValueError("config index must be 1..5")
@@ -393,7 +396,7 @@ def make_config(idx: int, seed: Optional[int] = None, with_logits: bool = True, 
     if with_logits:
         t.logits, t.draft_ids, t.match_len = fill_logits_and_drafts(batch, rng, p_geo)
     t.verdict = fill_verdicts(batch, rng, p_ver)
-    recipe = {"p_mismatch": p_geo, "p_step_accept": p_ver, "poison": poison}
+    recipe = {"p_mismatch": p_geo, "p_step_accept": p_ver, "poison": poison, "carry_in": carry_in}
     return Workload(CONFIG_NAMES[idx], seed, batch, t, recipe)
 
 

@@ -36,6 +36,14 @@ def test_whole_pass_full_size_configs(cfg):
     run_and_check_pass(make_config(cfg))
 
 
+@pytest.mark.parametrize("cfg", [1, 2, 5])
+def test_whole_pass_with_the_carry_in_token_as_a_query(cfg):
+    """q_len = L + 1: the last accepted token and the L drafts are the queries, one per logits row."""
+    w = make_config(cfg, carry_in=True)
+    assert w.batch.n_q_rows == w.batch.n_logit_rows
+    run_and_check_pass(w)
+
+
 @pytest.mark.parametrize("seed", list(range(16)))
 def test_whole_pass_ragged_small(seed):
     run_and_check_pass(make_random_small(1000 + seed))
