@@ -26,6 +26,8 @@ What is computed, and where the paper fixes it:
   probability min(1, P/Q) and a final token from the residual distribution, for point-mass draft
   distributions (prompt-lookup drafts, the paper's SD method), temperature sampling, random numbers
   passed in.
+* ``compact``           -- the step after the output construction: the committed sequence, scattered
+  over partly filled pages, rewritten densely into its leading kept pages (no arithmetic on values).
 * ``commit``            -- Algorithm 1, last two lines: j* = min({j : V(s_j, s^_j)
   = False} U {gamma}); output = s^_0 .. s^_{j*-1} (+) s_{j*}.  On the KV cache
   this keeps the prefix pages, the pages of the first j* segments and the pages
@@ -302,6 +304,35 @@ def accept_sample(logits_bits: np.ndarray, draft_ids: np.ndarray, cu_draft: np.n
         n_accept[b] = n
         final_id[b] = sample_inverse_cdf(residual, float(u_final[b]))
     return n_accept, final_id, p_draft
+
+
+# ---------------------------------------------------------------------------
+# a3'. compaction of the committed KV (the step after commit)
+# ---------------------------------------------------------------------------
+def compact(keep_off: np.ndarray, keep_pages: np.ndarray, keep_valid: np.ndarray, k_pool_bits: np.ndarray,
+            v_pool_bits: np.ndarray):
+    """After the output construction of Algorithm 1 the committed sequence of a request lies in its kept
+    pages, some of them partly filled (the last page of the prefix, of every accepted segment and of the
+    kept tail).  Compaction rewrites it densely: token k of the committed sequence goes to slot k % 16 of
+    the request's kept page number k // 16, so that the sequence is one span again (the shared prefix of
+    the next cycle).  Returns (new_len, n_pages_kept, k_pool, v_pool): per request its length and the number
+    of leading pages of its keep list that now hold it (the rest of the list is no longer needed); the
+    pools are modified copies.  Bytes outside the first new_len tokens of those pages are unspecified.
+    """
+    R = len(keep_off) - 1
+    k_out, v_out = k_pool_bits.copy(), v_pool_bits.copy()
+    new_len = np.zeros(R, dtype=np.int32)
+    n_kept = np.zeros(R, dtype=np.int32)
+    for r in range(R):
+        pages = [int(p) for p in keep_pages[keep_off[r] : keep_off[r + 1]]]
+        valid = [int(v) for v in keep_valid[keep_off[r] : keep_off[r + 1]]]
+        seq = [(pg, t) for pg, v in zip(pages, valid) for t in range(v)]  # committed tokens in order
+        for k, (pg, t) in enumerate(seq):  # read from the ORIGINAL pools: the moves do not see each other
+            k_out[pages[k // PAGE], :, k % PAGE, :] = k_pool_bits[pg, :, t, :]
+            v_out[pages[k // PAGE], :, k % PAGE, :] = v_pool_bits[pg, :, t, :]
+        new_len[r] = len(seq)
+        n_kept[r] = (len(seq) + PAGE - 1) // PAGE
+    return new_len, n_kept, k_out, v_out
 
 
 def verify_pass(batch, q_bits, k_pool_bits, v_pool_bits, logits_bits, draft_ids, verdict):
