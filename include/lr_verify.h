@@ -251,6 +251,26 @@ int lr_commit(lr_plan *plan, const uint8_t *verdict_d, const int32_t *n_accept_d
               int32_t *keep_off_d, int32_t *keep_pages_d, int32_t *keep_valid_d,
               int32_t *free_off_d, int32_t *free_pages_d, void *stream);
 
+/*
+ * Compaction of the committed KV (the step after the output construction of
+ * Algorithm 1: the accepted draft steps and the decisive target step become the
+ * shared context of the next cycle).  Input: the keep lists lr_commit wrote.
+ * Token k of request r's committed sequence is moved, in place in the pools, to
+ * slot k % 16 of the page keep_pages[keep_off[r] + k / 16].  Outputs per request:
+ * new_len = its committed length; n_pages_kept = ceil(new_len / 16): that many
+ * leading entries of its keep list now hold the sequence densely, the remaining
+ * entries of its keep list are no longer needed by it.  Tokens in front of the
+ * request's first partly filled kept page are not touched.  Bytes of the kept
+ * pages beyond the sequence are unspecified afterwards; no other page is written.
+ * scratch_d: lr_compact_scratch_bytes bytes, 256-byte aligned, no initial
+ * contents needed.  Three launches on `stream`; a page id outside the pools sets
+ * the plan's status word (LR_EBOUNDS) instead of being dereferenced.  The batch
+ * must be the one the plan and the keep lists were made for.
+ */
+int lr_compact_scratch_bytes(const lr_plan *plan, size_t *bytes_out);
+int lr_compact(lr_plan *plan, const int32_t *keep_off_d, const int32_t *keep_pages_d, const int32_t *keep_valid_d,
+               void *k_pool_d, void *v_pool_d, int32_t *new_len_d, int32_t *n_pages_kept_d, void *scratch_d, void *stream);
+
 /* ---- whole pass with host buffers ---------------------------------------- */
 
 /* Host-side inputs and outputs of one pass; every pointer is a HOST pointer

@@ -79,6 +79,8 @@ def lib() -> C.CDLL:
             "lr_accept_sample_scratch_bytes": [vp, i32, C.POINTER(sz)],
             "lr_accept_sample": [vp, vp, i64, vp, vp, i32, i32, f32, vp, vp, vp, vp, vp, vp, vp],
             "lr_commit": [vp] + [vp] * 10 + [vp],
+            "lr_compact_scratch_bytes": [vp, C.POINTER(sz)],
+            "lr_compact": [vp] * 10,
             "lr_pass_staging_bytes": [vp, C.POINTER(sz)],
             "lr_verify_pass_host": [vp, C.POINTER(lr_pass_host_io), vp, vp, vp, sz, f32, vp],
             "lr_poll_status": [vp, vp, C.POINTER(i32)],
@@ -254,6 +256,18 @@ class Plan:
         _check(lib().lr_commit(self.handle, _ptr(verdict), _ptr(n_accept), _ptr(n_steps_accepted), _ptr(survivor),
                                _ptr(committed_len), _ptr(keep_off), _ptr(keep_pages), _ptr(keep_valid), _ptr(free_off),
                                _ptr(free_pages), _stream_ptr(stream)), "lr_commit")
+
+    def compact_scratch(self) -> torch.Tensor:
+        n = C.c_size_t()
+        _check(lib().lr_compact_scratch_bytes(self.handle, C.byref(n)), "lr_compact_scratch_bytes")
+        t = torch.empty(n.value + 256, dtype=torch.uint8, device=f"cuda:{self.ctx.device}")
+        off = (-t.data_ptr()) % 256
+        return t[off : off + n.value]
+
+    def lr_compact(self, keep_off, keep_pages, keep_valid, k_pool, v_pool, new_len, n_pages_kept, scratch, stream=None) -> None:
+        """Moves the committed tokens (keep lists of ``lr_commit``) densely into the leading kept pages, in place."""
+        _check(lib().lr_compact(self.handle, _ptr(keep_off), _ptr(keep_pages), _ptr(keep_valid), _ptr(k_pool), _ptr(v_pool),
+                                _ptr(new_len), _ptr(n_pages_kept), _ptr(scratch), _stream_ptr(stream)), "lr_compact")
 
     def lr_poll_status(self, stream=None) -> int:
         d = C.c_int32()

@@ -98,7 +98,8 @@ static int validate_batch(const lr_batch *b) {
 struct Layout {
   Image img;
   size_t o_req_span_off, o_span_len, o_span_slot, o_br_req, o_br_depth, o_br_own_len, o_br_own_slot, o_br_n_draft, o_cu_q,
-      o_cu_draft, o_page_ids, o_req_br_off, o_span_req, o_status, o_slot_item, o_chain_pg, o_chain_tok, o_tail_pg;
+      o_cu_draft, o_page_ids, o_req_br_off, o_span_req, o_status, o_slot_item, o_chain_pg, o_chain_tok, o_tail_pg, o_compact_stage_off;
+  size_t compact_tokens;
   std::vector<int32_t> cu_draft;
   TcHostPlan tc;
   size_t image_bytes, total_bytes;
@@ -156,6 +157,19 @@ static int build_layout(const lr_ctx *ctx, const lr_batch *b, Layout &L) {
     L.o_chain_pg = g.add(chain_pg.data(), I * chain_pg.size());
     L.o_chain_tok = g.add(chain_tok.data(), I * chain_tok.size());
     L.o_tail_pg = g.add(tail_pg.data(), I * tail_pg.size());
+    // lr_compact: at most the segments and one tail of a request are displaced
+    std::vector<int32_t> stage_off((size_t)b->n_req + 1, 0);
+    size_t tokens = 0;
+    for (int r = 0; r < b->n_req; ++r) {
+      stage_off[r] = (int32_t)tokens;
+      size_t segs = 0, tail = 0;
+      for (int s = b->req_span_off[r] + 1; s < b->req_span_off[r + 1]; ++s) segs += (size_t)b->span_len[s];
+      for (int i = req_br_off[r]; i < req_br_off[r + 1]; ++i) tail = std::max(tail, (size_t)b->br_own_len[i]);
+      tokens += segs + tail;
+      stage_off[r + 1] = (int32_t)tokens;
+    }
+    L.compact_tokens = tokens;
+    L.o_compact_stage_off = g.add(stage_off.data(), I * stage_off.size());
   }
   int32_t zero2[2] = {0, 0};
   L.o_status = g.add(zero2, sizeof(zero2));
@@ -297,6 +311,15 @@ extern "C" int lr_plan_create(lr_ctx *ctx, const lr_batch *b, void *ws, size_t w
   d.chain_pg = at(L.o_chain_pg);
   d.chain_tok = at(L.o_chain_tok);
   d.tail_pg = at(L.o_tail_pg);
+  d.compact_stage_off = at(L.o_compact_stage_off);
+  {
+    size_t off = 0;
+    auto take = [&](size_t n) { size_t o = off; off = align_up(off + n, 256); return o; };
+    p->compact.o_tok_off = take(sizeof(int32_t) * (size_t)b->n_page_slots);
+    p->compact.o_first_moved = take(sizeof(int32_t) * (size_t)b->n_req);
+    p->compact.o_staging = take(L.compact_tokens * 2 * (size_t)ctx->model.n_kv_heads * ctx->model.head_dim * 2);
+    p->compact.bytes = std::max<size_t>(off, 256);
+  }
   d.status = reinterpret_cast<int32_t *>(base + L.o_status);
   d.n_req = b->n_req;
   d.n_branch = b->n_branch;
@@ -460,6 +483,29 @@ extern "C" int lr_commit(lr_plan *p, const uint8_t *verdict, const int32_t *n_ac
   }
   return launch_commit(p, verdict, n_accept, n_steps, survivor, committed, keep_off, keep_pages, keep_valid, free_off,
                        free_pages, reinterpret_cast<cudaStream_t>(stream));
+}
+
+extern "C" int lr_compact_scratch_bytes(const lr_plan *p, size_t *bytes_out) {
+  if (!p || !bytes_out) {
+    set_error("lr_compact_scratch_bytes: null argument");
+    return LR_EINVAL;
+  }
+  *bytes_out = p->compact.bytes;
+  return LR_OK;
+}
+
+extern "C" int lr_compact(lr_plan *p, const int32_t *keep_off, const int32_t *keep_pages, const int32_t *keep_valid, void *k_pool,
+                          void *v_pool, int32_t *new_len, int32_t *n_pages_kept, void *scratch, void *stream) {
+  if (!p || !keep_off || !keep_pages || !keep_valid || !k_pool || !v_pool || !new_len || !n_pages_kept || !scratch) {
+    set_error("lr_compact: null argument");
+    return LR_EINVAL;
+  }
+  if ((((uintptr_t)k_pool | (uintptr_t)v_pool) & 15) != 0 || ((uintptr_t)scratch & 255) != 0) {
+    set_error("lr_compact: pools must be 16-byte aligned and the scratch 256-byte aligned");
+    return LR_EINVAL;
+  }
+  return launch_compact(p, keep_off, keep_pages, keep_valid, k_pool, v_pool, new_len, n_pages_kept, scratch,
+                        reinterpret_cast<cudaStream_t>(stream));
 }
 
 // ---- status --------------------------------------------------------------------

@@ -35,6 +35,7 @@ struct DevBatch {
   const int32_t *chain_pg;    // [n_span + n_req]
   const int32_t *chain_tok;   // [n_span + n_req]
   const int32_t *tail_pg;     // [n_branch + n_req]
+  const int32_t *compact_stage_off;  // [n_req+1] staging-token range of each request in lr_compact
   int32_t n_req, n_branch, n_span, n_page_slots, n_q_rows;
   int32_t n_q_heads, n_kv_heads, head_dim, group;
   int64_t n_pool_pages;
@@ -122,6 +123,7 @@ struct lr_plan {
   size_t image_bytes;
   void *workspace_d;
   size_t workspace_bytes;
+  struct { size_t o_tok_off, o_first_moved, o_staging, bytes; } compact;  // layout of lr_compact's scratch
   // host copies needed at launch time
   int32_t n_rows_logits, n_drafts, n_verdicts;
   std::vector<int32_t> cu_draft_h;
@@ -172,6 +174,8 @@ size_t accept_sample_scratch_bytes(int32_t vocab, int32_t n_rows);
 int launch_accept_sample(lr_ctx *ctx, const void *logits, int64_t stride, const int32_t *drafts, const int32_t *cu_draft,
                          int32_t n_branch, int32_t n_rows, float temperature, const float *u_accept, const float *u_final,
                          int32_t *n_accept, int32_t *final_id, float *p_draft, void *scratch, cudaStream_t s);
+int launch_compact(lr_plan *p, const int32_t *keep_off, const int32_t *keep_pages, const int32_t *keep_valid, void *k_pool,
+                   void *v_pool, int32_t *new_len, int32_t *n_pages_kept, void *scratch, cudaStream_t s);
 int launch_commit(lr_plan *p, const uint8_t *verdict, const int32_t *n_accept, int32_t *n_steps, int32_t *survivor,
                   int32_t *committed, int32_t *keep_off, int32_t *keep_pages, int32_t *keep_valid, int32_t *free_off,
                   int32_t *free_pages, cudaStream_t s);
