@@ -280,6 +280,23 @@ def main():
     def sample_only(c):
         ctx.lr_accept_sample(lc[c], x0.draft_ids, x0.cu_draft, 0.6, u_acc, u_fin, samp_n, samp_f, samp_scratch, None, None)
 
+    # compaction of the committed KV (not part of the timed step), timed alone on two pool copies of its own: it moves
+    # tokens in place, and every call with the same keep lists moves the same number of bytes
+    cmp_k = [x0.k_pool.clone() for _ in range(2)]
+    cmp_v = [x0.v_pool.clone() for _ in range(2)]
+    cmp_scratch = plan.compact_scratch()
+    cmp_len = torch.empty(b.n_req, dtype=torch.int32, device=dev)
+    cmp_kept = torch.empty(b.n_req, dtype=torch.int32, device=dev)
+
+    # keep lists of the commit that displaces the most: every step accepted, every draft token of the last branch kept
+    yc = R.PassOutputs(b, dev, n_rows=1)
+    plan.lr_commit(torch.ones_like(x0.verdict), torch.from_numpy(np.ascontiguousarray(b.br_n_draft, dtype=np.int32)).to(dev),
+                   yc.n_steps_accepted, yc.survivor, yc.committed_len, yc.keep_off, yc.keep_pages, yc.keep_valid,
+                   yc.free_off, yc.free_pages, None)
+
+    def compact_only(c):
+        plan.lr_compact(yc.keep_off, yc.keep_pages, yc.keep_valid, cmp_k[c % 2], cmp_v[c % 2], cmp_len, cmp_kept, cmp_scratch, None)
+
     def make_runner(fn):
         """Returns run(first, count): `count` consecutive calls fn(i % copies) starting at index `first`."""
         graph = None
@@ -317,6 +334,7 @@ def main():
     run_accept, _ = make_runner(accept_only)
     run_commit, _ = make_runner(commit_only)
     run_sample, _ = make_runner(sample_only)
+    run_compact, _ = make_runner(compact_only)
     torch.cuda.synchronize()
     run_step(0, copies)  # one replay as warm-up of the graph itself
     assert plan.lr_poll_status() == 0
@@ -343,7 +361,8 @@ def main():
 
     # ---- region B: each kernel alone, K back-to-back launches over the rotating copies ------
     kernel_us = {"attention": 1e3 * timed(run_attn, K) / K, "accept": 1e3 * timed(run_accept, K) / K,
-                 "commit": 1e3 * timed(run_commit, K) / K, "sample": 1e3 * timed(run_sample, K) / K}
+                 "commit": 1e3 * timed(run_commit, K) / K, "sample": 1e3 * timed(run_sample, K) / K,
+                 "compact": 1e3 * timed(run_compact, K) / K}
     clocks = sampler.stop() if rank == 0 else None
     assert plan.lr_poll_status() == 0
 
@@ -416,6 +435,18 @@ def main():
                                  "algorithmic_bytes": acc_b, "temperature": 0.6,
                                  "note": "rejection-sampling acceptance; not part of the timed step"},
         }
+        # tokens lr_compact displaces: those behind the first partly filled kept page of each request
+        k_off, k_val = yc.keep_off.cpu().numpy(), yc.keep_valid.cpu().numpy()
+        displaced = 0
+        for r in range(b.n_req):
+            v = k_val[k_off[r]:k_off[r + 1]]
+            partial = np.flatnonzero(v[:-1] != 16)
+            if len(partial):
+                displaced += int(v[partial[0] + 1:].sum())
+        cmp_bytes = displaced * 2 * b.model.n_kv_heads * b.model.head_dim * 2 * 4  # K and V, read and written, twice
+        kernels["lr_compact"] = {"us": kernel_us["compact"], "displaced_tokens": displaced, "bytes_moved": cmp_bytes,
+                                 "case": "all steps accepted, whole last draft kept",
+                                 "note": "three dependent launches, latency-bound; not part of the timed step"}
         cpu = None
         if not args.no_cpu_baseline:
             sec, n = oracle_pass_seconds(w, args.cpu_seconds)
