@@ -20,4 +20,6 @@ from .gen import (  # noqa: F401
     fill_verdicts,
     make_config,
     make_random_small,
+    make_tree,
+    make_random_tree,
 )

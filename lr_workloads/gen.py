@@ -90,6 +90,10 @@ class Batch:
     cu_q: np.ndarray  # [B+1] query-row offsets
     page_ids: np.ndarray  # [n_page_slots] physical page numbers
     n_pool_pages: int
+    # Multi-branch (tree) drafting: [n_span], for segment c of a request the local index (0 = prefix, else an
+    # earlier segment) of the segment it continues; -1 at the prefix spans.  None = the nested chain (parent c - 1).
+    # With a tree, br_depth[b] is the local index of the node branch b continues (0 = the prefix alone).
+    seg_parent: Optional[np.ndarray] = None
 
     @property
     def n_req(self) -> int:
@@ -170,7 +174,8 @@ def build_batch(
 ) -> Batch:
     """Lay out page slots and tables.
 
-    ``requests[r]`` = ``{"P": int, "segs": [len...], "branches": [(depth, own_len, q_len, n_draft), ...]}``.
+    ``requests[r]`` = ``{"P": int, "segs": [len...], "branches": [(depth, own_len, q_len, n_draft), ...]}``,
+    plus ``"parents": [parent of segment 1, ...]`` (0 = prefix) when any request is a tree.
     Every span (prefix, segment, tail) owns whole pages and starts at slot 0 of
     its first page; a physical page belongs to at most one span.
     """
@@ -184,7 +189,10 @@ def build_batch(
     br_n_draft: List[int] = []
     cu_q = [0]
     slot = 0
+    tree = any("parents" in req for req in requests)
+    seg_parent: List[int] = []
     for r, req in enumerate(requests):
+        seg_parent += [-1] + [int(v) for v in req.get("parents", range(len(req["segs"])))]
         for ln in [req["P"]] + list(req["segs"]):
             span_len.append(int(ln))
             span_slot.append(slot)
@@ -218,6 +226,7 @@ def build_batch(
         cu_q=i32(cu_q),
         page_ids=page_ids,
         n_pool_pages=n_pool,
+        seg_parent=i32(seg_parent) if tree else None,
     )
 
 
@@ -439,3 +448,86 @@ def make_random_small(seed: int, head_dim: Optional[int] = None, max_prefix: int
     t.logits, t.draft_ids, t.match_len = fill_logits_and_drafts(batch, rng, 0.3)
     t.verdict = fill_verdicts(batch, rng, 0.6)
     return Workload(f"random_small_{seed}", seed, batch, t, {"p_mismatch": 0.3, "p_step_accept": 0.6})
+
+
+# --------------------------------------------------------------------------
+# multi-branch (tree) drafting
+# --------------------------------------------------------------------------
+def _tree_request(P: int, W: int, gamma: int, seg_len, L: int) -> dict:
+    """Full W-ary tree of draft steps, gamma levels deep, numbered level by level (so a parent precedes its
+    children); one branch per node, the prefix alone included: the target continues every draft prefix."""
+    parents: List[int] = []
+    level = [0]
+    for _ in range(gamma):
+        nxt = []
+        for node in level:
+            for _ in range(W):
+                parents.append(node)
+                nxt.append(len(parents))
+        level = nxt
+    segs = [int(seg_len(i)) for i in range(len(parents))]
+    return {"P": P, "segs": segs, "parents": parents, "branches": [(n, L, L, L) for n in range(len(parents) + 1)]}
+
+
+def _finish(name: str, seed: int, model: Model, reqs, rng, p_geo: float, p_ver: float, with_logits: bool,
+            with_kv: bool, poison: str) -> Workload:
+    batch = build_batch(model, reqs, rng, shuffle=True)
+    t = Tensors()
+    if with_kv:
+        k_scale = rng.uniform(0.5, 2.0, size=(batch.n_req, model.n_kv_heads)).astype(np.float32)
+        t.k_pool, t.v_pool = fill_kv(batch, rng, k_head_scale=k_scale, poison=poison)
+        t.q = fill_q(batch, rng)
+    if with_logits:
+        t.logits, t.draft_ids, t.match_len = fill_logits_and_drafts(batch, rng, p_geo)
+    t.verdict = fill_verdicts(batch, rng, p_ver)
+    return Workload(name, seed, batch, t, {"p_mismatch": p_geo, "p_step_accept": p_ver, "poison": poison})
+
+
+def make_tree(W: int, gamma: int, seed: Optional[int] = None, size: str = "layer", with_logits: bool = True,
+              with_kv: bool = True, poison: str = "nan") -> Workload:
+    """Tree-drafting workloads.  ``size`` "tiny": the geometry of config 1 (prefix 250, ragged segments);
+    "layer": the geometry of config 2 (one request, prefix 4096, segments of 32, L = 16);
+    "serving": 8 requests with the ragged lengths of config 5."""
+    if seed is None:
+        seed = 20250700 + 16 * W + gamma
+    rng = np.random.Generator(np.random.PCG64(seed))
+    if size == "tiny":
+        model = Model(4, 1, 64, 1024)
+        reqs = [_tree_request(250, W, gamma, lambda i: rng.integers(5, 40), 8)]
+    elif size == "layer":
+        model = Model(40, 8, 128, 152064)
+        reqs = [_tree_request(4096, W, gamma, lambda i: 32, 16)]
+    elif size == "serving":
+        model = Model(40, 8, 128, 152064)
+        reqs = [_tree_request(int(rng.integers(1024, 16384 + 1)), W, gamma, lambda i: rng.integers(16, 64 + 1),
+                              int(rng.choice([4, 8, 16]))) for _ in range(8)]
+    else:
+        raise ValueError("size must be tiny, layer or serving")
+    return _finish(f"tree_w{W}_g{gamma}_{size}", seed, model, reqs, rng, 0.25, 0.6, with_logits, with_kv, poison)
+
+
+def make_random_tree(seed: int, head_dim: Optional[int] = None, poison: str = "nan", max_nodes: int = 9) -> Workload:
+    """Small ragged batches of irregular trees: every segment picks any earlier node as its parent (so chains,
+    stars and everything between occur), branches hang off arbitrary nodes, some nodes have none, some several;
+    one request in three is a plain chain written as a tree."""
+    rng = np.random.Generator(np.random.PCG64(seed))
+    if head_dim is None:
+        head_dim = int(rng.choice([64, 128]))
+    h_kv = int(rng.choice([1, 2]))
+    group = int(rng.choice([1, 2, 4, 5, 8]))
+    model = Model(h_kv * group, h_kv, head_dim, int(rng.choice([1000, 1024, 4099])))
+    reqs = []
+    for _ in range(int(rng.integers(1, 4))):
+        P = int(rng.choice([0, 1, 16, 17, int(rng.integers(0, 201))]))
+        n = int(rng.integers(0, max_nodes + 1))
+        chain = rng.random() < 1 / 3
+        parents = [c if chain else int(rng.integers(0, c + 1)) for c in range(n)]
+        segs = [int(v) for v in rng.integers(1, 41, size=n)]
+        branches = []
+        for _ in range(int(rng.integers(1, n + 3))):
+            q_len = int(rng.integers(1, 10))
+            own_len = q_len + int(rng.choice([0, 0, 1, 7, 20]))
+            n_draft = min(own_len, int(rng.choice([q_len, max(1, q_len - 1), int(rng.integers(1, 9))])))
+            branches.append((int(rng.integers(0, n + 1)), own_len, q_len, n_draft))
+        reqs.append({"P": P, "segs": segs, "parents": parents, "branches": branches})
+    return _finish(f"random_tree_{seed}", seed, model, reqs, rng, 0.3, 0.6, True, True, poison)

@@ -62,12 +62,29 @@ def bf16_bits_to_f64(u: np.ndarray) -> np.ndarray:
 # ---------------------------------------------------------------------------
 # a1. nested-prefix attention
 # ---------------------------------------------------------------------------
+def node_path(batch, r: int, node: int) -> List[int]:
+    """Draft steps (local span indices of request ``r``) between the prefix and ``node``, ``node`` included, in
+    sequence order.  On the nested chain of Algorithm 1 that is 1..node.  With multi-branch drafting (Section 3,
+    "Multi-Branch Drafting") every draft step continues one earlier step, or the prefix, named by ``seg_parent``;
+    the draft prefix of a node is then the steps met walking up to the prefix, reversed."""
+    parent = getattr(batch, "seg_parent", None)
+    if parent is None:
+        return list(range(1, node + 1))
+    s0 = int(batch.req_span_off[r])
+    up = []
+    while node != 0:
+        up.append(node)
+        node = int(parent[s0 + node])
+    return up[::-1]
+
+
 def branch_token_table(batch, b: int) -> Tuple[np.ndarray, np.ndarray, int]:
     """Physical (page, in-page offset) of every token branch ``b`` can ever see, in
-    sequence order: prefix, segments 1..depth, then its own tail.  Returns
+    sequence order: prefix, the draft steps in front of it, then its own tail.  Returns
     (pages, offsets, N_b) with N_b the number of chain tokens (prefix+segments).
 
-    Follows x'_j = x_{1:t} (+) s^_0..s^_{j-1} (Algorithm 1) with j = depth.
+    Follows x'_j = x_{1:t} (+) s^_0..s^_{j-1} (Algorithm 1) with j = depth; with a tree of
+    draft steps the steps are those on the way to the node the branch continues.
     """
     r = int(batch.br_req[b])
     s0 = int(batch.req_span_off[r])
@@ -80,7 +97,7 @@ def branch_token_table(batch, b: int) -> Tuple[np.ndarray, np.ndarray, int]:
         pages.append(np.asarray(batch.page_ids)[first_slot + t // PAGE].astype(np.int64))
         offs.append(t % PAGE)
 
-    for c in range(depth + 1):  # span 0 is the prefix, span c is segment c
+    for c in [0] + node_path(batch, r, depth):  # span 0 is the prefix, span c is segment c
         walk(int(batch.span_slot[s0 + c]), int(batch.span_len[s0 + c]))
     n_chain = int(sum(len(p) for p in pages))
     walk(int(batch.br_own_slot[b]), int(batch.br_own_len[b]))
@@ -184,6 +201,8 @@ def commit(batch, verdict: np.ndarray, n_accept: np.ndarray):
     free order: pages of segments j*+1..gamma, then branch tails in branch order
     (for the decisive branch only the pages past its kept ones).
     """
+    if getattr(batch, "seg_parent", None) is not None:
+        return _commit_tree(batch, verdict, n_accept)
     R = batch.n_req
     cu_v = batch.cu_verdict
     cu_d = batch.cu_draft
@@ -246,6 +265,74 @@ def commit(batch, verdict: np.ndarray, n_accept: np.ndarray):
         "free_off": i32(free_off),
         "free_pages": i32(free_pages),
     }
+
+
+def _commit_tree(batch, verdict: np.ndarray, n_accept: np.ndarray):
+    """Commit with multi-branch drafting (Section 3, "Multi-Branch Drafting").
+
+    Verdict c - 1 of a request says whether draft step c agrees with the step the target wrote as the
+    continuation of c's parent.  Starting at the prefix, the walk moves to a child whose verdict is True -- the
+    lowest-numbered one if several agree; the others are discarded -- and stops where no child agrees.  j* is the
+    number of moves, the decisive target step is the branch that continues the node where the walk stopped
+    (lowest index; -1 if none), and the kept KV is the prefix, the steps walked through and that branch's
+    kept tail.  Lists: keep in sequence order; free = every other draft step in index order, then the tails in
+    branch order (the decisive branch: only pages past its kept ones).  On a chain this is Algorithm 1's rule.
+    """
+    R = batch.n_req
+    cu_v, cu_d = batch.cu_verdict, batch.cu_draft
+    out = {k: [] for k in ("n_steps_accepted", "survivor", "committed_len")}
+    keep_off, free_off = [0], [0]
+    keep_pages: List[int] = []
+    keep_valid: List[int] = []
+    free_pages: List[int] = []
+
+    def span_pages(first_slot: int, n_tok: int):
+        npg = (n_tok + PAGE - 1) // PAGE
+        return [(int(batch.page_ids[first_slot + p]), min(PAGE, n_tok - p * PAGE)) for p in range(npg)]
+
+    for r in range(R):
+        s0, s1 = int(batch.req_span_off[r]), int(batch.req_span_off[r + 1])
+        n_seg = s1 - s0 - 1
+        node, walked = 0, []
+        while True:
+            agreeing = [c for c in range(1, n_seg + 1)
+                        if int(batch.seg_parent[s0 + c]) == node and bool(verdict[cu_v[r] + c - 1])]
+            if not agreeing:
+                break
+            node = agreeing[0]
+            walked.append(node)
+        branches = [b for b in range(batch.n_branch) if int(batch.br_req[b]) == r]
+        decisive = [b for b in branches if int(batch.br_depth[b]) == node]
+        s = decisive[0] if decisive else -1
+        length = 0
+        for c in [0] + walked:
+            ln = int(batch.span_len[s0 + c])
+            length += ln
+            for pg, val in span_pages(int(batch.span_slot[s0 + c]), ln):
+                keep_pages.append(pg)
+                keep_valid.append(val)
+        kept_tail = 0
+        if s >= 0:
+            kept_tail = int(batch.br_own_len[s]) - int(cu_d[s + 1] - cu_d[s]) + int(n_accept[s])
+            length += kept_tail
+            for pg, val in span_pages(int(batch.br_own_slot[s]), kept_tail):
+                keep_pages.append(pg)
+                keep_valid.append(val)
+        for c in range(1, n_seg + 1):
+            if c not in walked:
+                free_pages += [pg for pg, _ in span_pages(int(batch.span_slot[s0 + c]), int(batch.span_len[s0 + c]))]
+        for b in branches:
+            pages = span_pages(int(batch.br_own_slot[b]), int(batch.br_own_len[b]))
+            skip = (kept_tail + PAGE - 1) // PAGE if b == s else 0
+            free_pages += [pg for pg, _ in pages[skip:]]
+        out["n_steps_accepted"].append(len(walked))
+        out["survivor"].append(s)
+        out["committed_len"].append(length)
+        keep_off.append(len(keep_pages))
+        free_off.append(len(free_pages))
+    i32 = lambda a: np.asarray(a, dtype=np.int32)  # noqa: E731
+    return {**{k: i32(v) for k, v in out.items()}, "keep_off": i32(keep_off), "keep_pages": i32(keep_pages),
+            "keep_valid": i32(keep_valid), "free_off": i32(free_off), "free_pages": i32(free_pages)}
 
 
 # ---------------------------------------------------------------------------
