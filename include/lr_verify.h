@@ -82,6 +82,17 @@ typedef struct lr_model {
  * br_own_len[b] tokens (slots from br_own_slot[b]); the LAST q_len_b =
  * cu_q[b+1]-cu_q[b] tail tokens are the queries.  br_n_draft[b] (<= own_len)
  * is L_b, the number of token-level drafts being verified for the branch.
+ *
+ * Multi-branch (tree) drafting (Section 3, "Multi-Branch Drafting"): with
+ * seg_parent != NULL the draft steps of a request form a tree.  For span s of
+ * request r, local index c = s - req_span_off[r] >= 1, seg_parent[s] is the
+ * local index (0 = the prefix, else 1..c-1) of the step that segment c
+ * continues; the entries at prefix spans are ignored.  br_depth[b] is then the
+ * local index of the node branch b continues (0 = the prefix alone): the
+ * branch sees the prefix and the segments on the way from the prefix to that
+ * node, in that order.  The nested chain is the tree with seg_parent = c - 1,
+ * and NULL means exactly that.  In tree mode no node may lie more than 8 steps
+ * below the prefix (LR_EINVAL otherwise).
  */
 typedef struct lr_batch {
   int32_t n_req, n_branch, n_span, n_page_slots;
@@ -96,6 +107,7 @@ typedef struct lr_batch {
   const int32_t *cu_q;         /* [n_branch+1] query-row offsets, q_len >= 1 */
   const int32_t *page_ids;     /* [n_page_slots] physical page numbers, distinct */
   int64_t n_pool_pages;        /* pages in each of the K and V pools */
+  const int32_t *seg_parent;   /* [n_span] or NULL (nested chain); see above */
 } lr_batch;
 
 /* Host-only check of a batch description against the rules above (no device
@@ -245,6 +257,15 @@ int lr_accept_greedy_static(lr_ctx *ctx, const void *logits_d, int64_t row_strid
  * then the branch tails in branch order (for the survivor only the pages past
  * the kept ones).  keep and free together list every page slot of the request
  * exactly once.  No KV data is moved.
+ *
+ * With a tree of draft steps (lr_batch.seg_parent; Section 3, "Multi-Branch
+ * Drafting") verdict c - 1 of a request says whether segment c agrees with the
+ * target step written after the node it continues.  Starting at the prefix the
+ * commit moves to the lowest-numbered child whose verdict is set, until no
+ * child agrees; n_steps_accepted is the number of moves, survivor the
+ * lowest-numbered branch that continues the node reached, the kept segments
+ * are those moved through (keep list in that order) and the free list holds
+ * every other segment in index order, then the tails as above.
  */
 int lr_commit(lr_plan *plan, const uint8_t *verdict_d, const int32_t *n_accept_d,
               int32_t *n_steps_accepted_d, int32_t *survivor_d, int32_t *committed_len_d,

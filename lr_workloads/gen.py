@@ -506,7 +506,7 @@ def make_tree(W: int, gamma: int, seed: Optional[int] = None, size: str = "layer
     return _finish(f"tree_w{W}_g{gamma}_{size}", seed, model, reqs, rng, 0.25, 0.6, with_logits, with_kv, poison)
 
 
-def make_random_tree(seed: int, head_dim: Optional[int] = None, poison: str = "nan", max_nodes: int = 9) -> Workload:
+def make_random_tree(seed: int, head_dim: Optional[int] = None, poison: str = "nan", max_nodes: int = 8) -> Workload:
     """Small ragged batches of irregular trees: every segment picks any earlier node as its parent (so chains,
     stars and everything between occur), branches hang off arbitrary nodes, some nodes have none, some several;
     one request in three is a plain chain written as a tree."""

@@ -42,7 +42,7 @@ class lr_batch(C.Structure):
         (n, _I32P)
         for n in ("req_span_off", "span_len", "span_slot", "br_req", "br_depth", "br_own_len", "br_own_slot",
                   "br_n_draft", "cu_q", "page_ids")
-    ] + [("n_pool_pages", C.c_int64)]
+    ] + [("n_pool_pages", C.c_int64), ("seg_parent", _I32P)]
 
 
 class lr_pass_host_io(C.Structure):
@@ -124,6 +124,10 @@ class HostBatch:
         for f in self.FIELDS:
             setattr(self.c, f, self.arrays[f].ctypes.data_as(_I32P))
         self.c.n_pool_pages = int(batch.n_pool_pages)
+        parent = getattr(batch, "seg_parent", None)  # tree of draft steps; absent = nested chain (NULL)
+        if parent is not None:
+            self.arrays["seg_parent"] = _i32(parent)
+            self.c.seg_parent = self.arrays["seg_parent"].ctypes.data_as(_I32P)
 
 
 def _model_struct(model) -> lr_model:

@@ -46,7 +46,8 @@ attn_generic_kernel(DevBatch d, const uint16_t *__restrict__ q, const uint16_t *
   }
   const int b = lo;
   const int i = row - d.cu_q[b], q_len = d.cu_q[b + 1] - d.cu_q[b];
-  const int depth = d.br_depth[b], s0 = d.req_span_off[d.br_req[b]];
+  const int s0 = d.req_span_off[d.br_req[b]], n_seg = d.req_span_off[d.br_req[b] + 1] - s0 - 1;
+  const int node = d.span_tin[s0 + d.br_depth[b]];  // depth-first number of the node the branch continues
   const int tail_vis = d.br_own_len[b] - q_len + i + 1;  // the query sees itself
 
   const uint16_t *qp = q + ((int64_t)row * d.n_q_heads + h) * D;
@@ -57,9 +58,10 @@ attn_generic_kernel(DevBatch d, const uint16_t *__restrict__ q, const uint16_t *
 #pragma unroll
   for (int e = 0; e < EPL; ++e) acc[e] = 0.f;
 
-  for (int sp = 0; sp <= depth + 1; ++sp) {
-    const int slot0 = (sp <= depth) ? d.span_slot[s0 + sp] : d.br_own_slot[b];
-    const int len = (sp <= depth) ? d.span_len[s0 + sp] : tail_vis;
+  for (int sp = 0; sp <= n_seg + 1; ++sp) {  // prefix, the segments the node descends from (index order), tail
+    if (sp <= n_seg && (node < d.span_tin[s0 + sp] || node > d.span_last[s0 + sp])) continue;
+    const int slot0 = (sp <= n_seg) ? d.span_slot[s0 + sp] : d.br_own_slot[b];
+    const int len = (sp <= n_seg) ? d.span_len[s0 + sp] : tail_vis;
     for (int t0 = 0; t0 < len; t0 += 32) {
       const int t = t0 + lane;
       bool valid = t < len;

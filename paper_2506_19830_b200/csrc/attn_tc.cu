@@ -43,9 +43,12 @@
 // occupies the first 64 columns of S_s.
 //
 // Visibility.  Tiles made only of full prefix pages need no mask.  In every other
-// tile each page carries (valid tokens, minimum depth, owning branch, tail
-// offset) and every row carries (depth, branch, causal limit): a row sees the
-// first n_ok tokens of a page, with n_ok from those six numbers.  V rows of
+// tile each page carries (valid tokens, first and last node number that sees it,
+// owning branch, tail offset) and every row carries (node number, branch, causal
+// limit): a row sees the first n_ok tokens of a page, with n_ok from those
+// numbers.  Node numbers are depth-first, so "the row's node descends from the
+// page's segment" is an interval test; on the nested chain the number is the
+// depth and the interval is [segment index, gamma].  V rows of
 // invalid token slots are zeroed in shared memory before the PV product so that
 // whatever the slack holds (NaN included) cannot reach the output.
 //
@@ -265,7 +268,7 @@ struct RingOrder {
 };
 
 struct RowInfo {
-  int depth;       // segments the row sees; -1 for padding rows
+  int depth;       // depth-first number of the node the row's branch continues (on a chain: segments it sees); -1 for padding rows
   int branch;      // local branch index within the request; -1 for padding rows
   int limit;       // last tail token the row sees
   int64_t q_index; // (query row * n_q_heads + head), -1 for padding rows
@@ -294,7 +297,7 @@ __device__ __forceinline__ RowInfo row_info(const DevBatch &d, const DevTcPlan &
 __device__ __forceinline__ int page_n_ok(uint32_t meta, const RowInfo &ri) {
   const int valid = meta & 31, need = (meta >> 5) & 255, owner = (meta >> 13) & 255, tb = meta >> 21;
   int n;
-  if (owner == 0) n = (ri.depth >= need) ? valid : 0;
+  if (owner == 0) n = (ri.depth >= need && ri.depth <= tb) ? valid : 0;  // the row's node lies in the span's subtree
   else n = (owner - 1 == ri.branch) ? min(valid, ri.limit - tb * kPage + 1) : 0;
   return max(n, 0);
 }
@@ -946,7 +949,8 @@ int init_attn_tc_kernel() {
 }
 
 // ---- host planning -----------------------------------------------------------------
-int tc_build_host_plan(const lr_ctx *ctx, const lr_batch *b, const int32_t *req_br_off, TcHostPlan &out, Image &img) {
+int tc_build_host_plan(const lr_ctx *ctx, const lr_batch *b, const int32_t *req_br_off, const int32_t *span_tin,
+                       const int32_t *span_last, TcHostPlan &out, Image &img) {
   out = TcHostPlan();
   const lr_model &m = ctx->model;
   const int G = m.n_q_heads / m.n_kv_heads;
@@ -969,31 +973,36 @@ int tc_build_host_plan(const lr_ctx *ctx, const lr_batch *b, const int32_t *req_
     if (br1 - br0 > 254) return LR_OK;
     rq.q_row0 = b->cu_q[br0];
     rq.n_q = b->cu_q[br1] - b->cu_q[br0];
-    int max_depth = 0;
+    std::vector<unsigned char> node_used((size_t)(s1 - s0), 0);  // by depth-first number: some branch continues it
     for (int i = br0; i < br1; ++i) {
-      max_depth = std::max(max_depth, b->br_depth[i]);
+      const int tin = span_tin[s0 + b->br_depth[i]];
+      node_used[tin] = 1;
       if ((b->br_own_len[i] + kPage - 1) / kPage > 2047) return LR_OK;
       const int q_len = b->cu_q[i + 1] - b->cu_q[i];
       for (int k = 0; k < q_len; ++k) {
         TcRow &w = rows[(size_t)b->cu_q[i] + k];
-        w.depth_branch = b->br_depth[i] | ((i - br0) << 16);
+        w.depth_branch = tin | ((i - br0) << 16);
         w.limit = b->br_own_len[i] - q_len + k;
       }
     }
-    auto add_span = [&](int slot, int len, int need, int owner) {
+    auto add_span = [&](int slot, int len, int need, int last, int owner) {
       const int n = (len + kPage - 1) / kPage;
       for (int p = 0; p < n; ++p) {
         TcPage e;
         e.page = b->page_ids[slot + p];
         const uint32_t valid = (uint32_t)std::min(kPage, len - p * kPage);
-        e.meta = valid | ((uint32_t)need << 5) | ((uint32_t)owner << 13) | ((uint32_t)(owner ? p : 0) << 21);
+        e.meta = valid | ((uint32_t)need << 5) | ((uint32_t)owner << 13) | ((uint32_t)(owner ? p : last) << 21);
         pages.push_back(e);
       }
     };
-    add_span(b->span_slot[s0], b->span_len[s0], 0, 0);
+    add_span(b->span_slot[s0], b->span_len[s0], 0, 255, 0);
     rq.n_dense_tiles = (b->span_len[s0] / kPage) / kPagesPerTile;
-    for (int c = 1; c <= max_depth && s0 + c < s1; ++c) add_span(b->span_slot[s0 + c], b->span_len[s0 + c], c, 0);
-    for (int i = br0; i < br1; ++i) add_span(b->br_own_slot[i], b->br_own_len[i], 0, i - br0 + 1);
+    for (int c = 1; s0 + c < s1; ++c) {  // a segment no branch sees is left out
+      bool seen = false;
+      for (int t = span_tin[s0 + c]; t <= span_last[s0 + c] && !seen; ++t) seen = node_used[t];
+      if (seen) add_span(b->span_slot[s0 + c], b->span_len[s0 + c], span_tin[s0 + c], span_last[s0 + c], 0);
+    }
+    for (int i = br0; i < br1; ++i) add_span(b->br_own_slot[i], b->br_own_len[i], 0, 0, i - br0 + 1);
     rq.n_pages = (int)pages.size() - rq.page_off;
     while (pages.size() % kPagesPerTile) pages.push_back(TcPage{0, 0});  // absent pages of the last tile: nothing valid
     const int n_tiles = (rq.n_pages + kPagesPerTile - 1) / kPagesPerTile;

@@ -167,9 +167,135 @@ commit_kernel(DevBatch d, const uint8_t *__restrict__ verdict,
   }
 }
 
+// Multi-branch drafting (Section 3, "Multi-Branch Drafting"): the draft steps form a tree and the kept steps are
+// those of a walk from the prefix that moves, at every node, to the lowest-numbered child whose verdict is set.
+// Same structure as commit_kernel; the walked nodes (at most kMaxTreeDepth, local indices below 256) are kept
+// as bytes in shared memory, and a page slot finds its place from the walk of its request.
+constexpr int kSmemPerReqTree = kSmemPerReq + kMaxTreeDepth;
+
+__global__ void __launch_bounds__(kThreads)
+commit_tree_kernel(DevBatch d, const uint8_t *__restrict__ verdict,
+                   const int32_t *__restrict__ n_accept, int32_t *__restrict__ n_steps_out, int32_t *__restrict__ survivor_out,
+                   int32_t *__restrict__ committed_out, int32_t *__restrict__ keep_off_out, int32_t *__restrict__ keep_pages,
+                   int32_t *__restrict__ keep_valid, int32_t *__restrict__ free_off_out, int32_t *__restrict__ free_pages) {
+  extern __shared__ int32_t sm[];
+  const int R = d.n_req;
+  int32_t *s_keep = sm, *s_free = sm + R, *s_a = sm + 2 * R, *s_surv = sm + 3 * R, *s_kp = sm + 4 * R, *s_kt = sm + 5 * R,
+          *s_kchain = sm + 6 * R;
+  uint8_t *s_walk = reinterpret_cast<uint8_t *>(sm + 7 * R);  // [R][kMaxTreeDepth]
+  __shared__ int32_t s_total[2];
+  const int tid = threadIdx.x;
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+
+  for (int r = tid; r < R; r += kThreads) {
+    const int s0 = d.req_span_off[r], s1 = d.req_span_off[r + 1];
+    const int b0 = d.req_br_off[r], b1 = d.req_br_off[r + 1];
+    const int n_seg = s1 - s0 - 1, base = s0 + r;
+    const uint8_t *v = verdict + (s0 - r);  // v[c - 1]: verdict of segment c
+    int node = 0, a = 0, kchain = d.chain_pg[base + 1], tokens = d.chain_tok[base + 1];
+    while (a < kMaxTreeDepth) {
+      int next = -1;
+      for (int k = d.child_off[s0 + node], k1 = d.child_off[s0 + node + 1]; k < k1 && next < 0; ++k) {
+        const int c = d.child_list[k];
+        if (v[c - 1] != 0) next = c;
+      }
+      if (next < 0) break;
+      s_walk[r * kMaxTreeDepth + a++] = (uint8_t)next;
+      node = next;
+      kchain += d.chain_pg[base + node + 1] - d.chain_pg[base + node];
+      tokens += d.chain_tok[base + node + 1] - d.chain_tok[base + node];
+    }
+    int surv = -1;  // lowest-numbered branch that continues the node where the walk stopped
+    for (int i = b0; i < b1 && surv < 0; ++i)
+      if (d.br_depth[i] == node) surv = i;
+    int kept_tail = 0;
+    if (surv >= 0) {
+      const int L = d.br_n_draft[surv], own = d.br_own_len[surv];
+      int na = n_accept[surv];
+      if (na < 0 || na > L) {
+        na = na < 0 ? 0 : L;
+        d.status[0] = kDevBounds;
+        d.status[1] = 301;
+      }
+      kept_tail = own - L + na;
+    }
+    const int chain_all = d.chain_pg[base + n_seg + 1], tails_all = d.tail_pg[b0 + r + (b1 - b0)];
+    const int kp = pages_of(kept_tail);
+    s_keep[r] = kchain + kp;
+    s_free[r] = chain_all + tails_all - kchain - kp;
+    s_a[r] = a;
+    s_surv[r] = surv;
+    s_kp[r] = kp;
+    s_kt[r] = kept_tail;
+    s_kchain[r] = kchain;
+    if (blockIdx.x == 0) {
+      n_steps_out[r] = a;
+      survivor_out[r] = surv;
+      committed_out[r] = tokens + kept_tail;
+    }
+  }
+  __syncthreads();
+  block_exclusive_scan(s_keep, R, &s_total[0]);
+  block_exclusive_scan(s_free, R, &s_total[1]);
+  if (blockIdx.x == 0) {
+    for (int r = tid; r < R; r += kThreads) {
+      keep_off_out[r] = s_keep[r];
+      free_off_out[r] = s_free[r];
+    }
+    if (tid == 0) {
+      keep_off_out[R] = s_total[0];
+      free_off_out[R] = s_total[1];
+    }
+  }
+
+  for (int i = blockIdx.x * kThreads + tid; i < d.n_page_slots; i += gridDim.x * kThreads) {
+    const int item = d.slot_item[i];
+    if (item < 0) continue;
+    const int32_t pid = d.page_ids[i];
+    if (item < d.n_span) {
+      const int s = item, r = d.span_req[s];
+      const int s0 = d.req_span_off[r], c = s - s0, a = s_a[r], base = s0 + r;
+      const int idx = i - d.span_slot[s];
+      // pages of walked segments numbered below c (walked indices increase), and whether c itself was walked
+      int walked_before = 0;
+      bool on_walk = c == 0;
+      for (int k = 0; k < a; ++k) {
+        const int w = s_walk[r * kMaxTreeDepth + k];
+        if (w < c) walked_before += d.chain_pg[base + w + 1] - d.chain_pg[base + w];
+        on_walk |= w == c;
+      }
+      if (on_walk) {
+        const int dst = s_keep[r] + (c == 0 ? 0 : d.chain_pg[base + 1] + walked_before) + idx;
+        keep_pages[dst] = pid;
+        keep_valid[dst] = min(kPage, d.span_len[s] - idx * kPage);
+      } else {
+        free_pages[s_free[r] + d.chain_pg[base + c] - d.chain_pg[base + 1] - walked_before + idx] = pid;
+      }
+    } else {
+      const int b = item - d.n_span, r = d.br_req[b];
+      const int s0 = d.req_span_off[r], s1 = d.req_span_off[r + 1], b0 = d.req_br_off[r];
+      const int surv = s_surv[r], kp = s_kp[r], kchain = s_kchain[r];
+      const int idx = i - d.br_own_slot[b];
+      if (b == surv && idx < kp) {
+        const int dst = s_keep[r] + kchain + idx;
+        keep_pages[dst] = pid;
+        keep_valid[dst] = min(kPage, s_kt[r] - idx * kPage);
+      } else {
+        const int chain_free = d.chain_pg[s0 + r + (s1 - s0)] - kchain;
+        const int tails_before = d.tail_pg[b0 + r + (b - b0)];
+        const int kept_before = (surv >= 0 && b >= surv) ? kp : 0;
+        free_pages[s_free[r] + chain_free + tails_before - kept_before + idx] = pid;
+      }
+    }
+  }
+}
+
 }  // namespace
 
 int init_commit_kernel() {
+  if (int rc = cuda_fail(cudaFuncSetAttribute(commit_tree_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              kMaxReq * kSmemPerReqTree), "commit_tree_kernel shared-memory attribute"))
+    return rc;
   return cuda_fail(cudaFuncSetAttribute(commit_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxReq * kSmemPerReq),
                    "commit_kernel shared-memory attribute");
 }
@@ -186,10 +312,15 @@ int launch_commit(lr_plan *p, const uint8_t *verdict, const int32_t *n_accept, i
   int grid = (d.n_page_slots + kThreads - 1) / kThreads;
   const int cap = d.n_req <= 64 ? 148 : (d.n_req <= 512 ? 32 : 8);
   grid = grid < 1 ? 1 : (grid > cap ? cap : grid);
+  p->ctx->launches++;
+  if (d.tree) {
+    commit_tree_kernel<<<grid, kThreads, (size_t)d.n_req * kSmemPerReqTree, s>>>(
+        d, verdict, n_accept, n_steps, survivor, committed, keep_off, keep_pages, keep_valid, free_off, free_pages);
+    return cuda_fail(cudaGetLastError(), "commit_tree_kernel launch");
+  }
   size_t smem = (size_t)d.n_req * kSmemPerReq;
   commit_kernel<<<grid, kThreads, smem, s>>>(d, verdict, n_accept, n_steps, survivor, committed,
                                               keep_off, keep_pages, keep_valid, free_off, free_pages);
-  p->ctx->launches++;
   return cuda_fail(cudaGetLastError(), "commit_kernel launch");
 }
 

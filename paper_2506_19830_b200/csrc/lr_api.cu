@@ -67,6 +67,16 @@ static int validate_batch(const lr_batch *b) {
       LR_REQUIRE(b->span_len[s] >= (s == s0 ? 0 : 1), "span %d of request %d has length %d", s - s0, r, b->span_len[s]);
       if (int rc = claim(b->span_slot[s], b->span_len[s], "span", s)) return rc;
     }
+    if (b->seg_parent) {
+      std::vector<int> level((size_t)(s1 - s0), 0);
+      for (int c = 1; c < s1 - s0; ++c) {
+        const int par = b->seg_parent[s0 + c];
+        LR_REQUIRE(par >= 0 && par < c, "request %d: segment %d continues %d, which is not the prefix or an earlier segment", r, c, par);
+        level[c] = level[par] + 1;
+        LR_REQUIRE(level[c] <= kMaxTreeDepth, "request %d: segment %d lies %d steps below the prefix (tree mode allows %d)", r,
+                   c, level[c], kMaxTreeDepth);
+      }
+    }
   }
   LR_REQUIRE(b->cu_q[0] == 0, "cu_q[0] must be 0");
   for (int i = 0; i < b->n_branch; ++i) {
@@ -98,7 +108,8 @@ static int validate_batch(const lr_batch *b) {
 struct Layout {
   Image img;
   size_t o_req_span_off, o_span_len, o_span_slot, o_br_req, o_br_depth, o_br_own_len, o_br_own_slot, o_br_n_draft, o_cu_q,
-      o_cu_draft, o_page_ids, o_req_br_off, o_span_req, o_status, o_slot_item, o_chain_pg, o_chain_tok, o_tail_pg, o_compact_stage_off;
+      o_cu_draft, o_page_ids, o_req_br_off, o_span_req, o_status, o_slot_item, o_chain_pg, o_chain_tok, o_tail_pg, o_compact_stage_off,
+      o_span_tin, o_span_last, o_child_off, o_child_list;
   size_t compact_tokens;
   std::vector<int32_t> cu_draft;
   TcHostPlan tc;
@@ -171,10 +182,40 @@ static int build_layout(const lr_ctx *ctx, const lr_batch *b, Layout &L) {
     L.compact_tokens = tokens;
     L.o_compact_stage_off = g.add(stage_off.data(), I * stage_off.size());
   }
+  // depth-first interval labels and child lists of the draft-step trees (a chain when seg_parent is absent)
+  std::vector<int32_t> span_tin((size_t)b->n_span, 0), span_last((size_t)b->n_span, 0), child_off((size_t)b->n_span + 1, 0),
+      child_list((size_t)b->n_span, 0);
+  for (int r = 0; r < b->n_req; ++r) {
+    const int s0 = b->req_span_off[r], n = b->req_span_off[r + 1] - s0;
+    auto parent_of = [&](int c) { return b->seg_parent ? b->seg_parent[s0 + c] : c - 1; };
+    std::vector<int> n_child((size_t)n, 0);
+    for (int c = 1; c < n; ++c) n_child[parent_of(c)]++;
+    for (int c = 0; c < n; ++c) child_off[s0 + c + 1] = child_off[s0 + c] + n_child[c];
+    std::vector<int> fill((size_t)n, 0);
+    for (int c = 1; c < n; ++c) {  // increasing c: every list comes out sorted
+      const int par = parent_of(c);
+      child_list[child_off[s0 + par] + fill[par]++] = c;
+    }
+    std::vector<int> size((size_t)n, 1);  // subtree sizes: children have larger indices than parents
+    for (int c = n - 1; c >= 1; --c) size[parent_of(c)] += size[c];
+    // pre-order numbers: a node's number is its parent's + 1 + the subtree sizes of its earlier siblings
+    for (int c = 0; c < n; ++c) {
+      int next = span_tin[s0 + c] + 1;
+      for (int k = child_off[s0 + c]; k < child_off[s0 + c + 1]; ++k) {
+        span_tin[s0 + child_list[k]] = next;
+        next += size[child_list[k]];
+      }
+      span_last[s0 + c] = span_tin[s0 + c] + size[c] - 1;
+    }
+  }
+  L.o_span_tin = g.add(span_tin.data(), I * span_tin.size());
+  L.o_span_last = g.add(span_last.data(), I * span_last.size());
+  L.o_child_off = g.add(child_off.data(), I * child_off.size());
+  L.o_child_list = g.add(child_list.data(), I * child_list.size());
   int32_t zero2[2] = {0, 0};
   L.o_status = g.add(zero2, sizeof(zero2));
   L.cu_draft = cu_draft;
-  if (int rc = tc_build_host_plan(ctx, b, req_br_off.data(), L.tc, g)) return rc;
+  if (int rc = tc_build_host_plan(ctx, b, req_br_off.data(), span_tin.data(), span_last.data(), L.tc, g)) return rc;
   L.image_bytes = align_up(g.bytes.size(), 256);
   L.total_bytes = L.image_bytes + align_up(L.tc.scratch_bytes, 256);
   return LR_OK;
@@ -312,6 +353,11 @@ extern "C" int lr_plan_create(lr_ctx *ctx, const lr_batch *b, void *ws, size_t w
   d.chain_tok = at(L.o_chain_tok);
   d.tail_pg = at(L.o_tail_pg);
   d.compact_stage_off = at(L.o_compact_stage_off);
+  d.span_tin = at(L.o_span_tin);
+  d.span_last = at(L.o_span_last);
+  d.child_off = at(L.o_child_off);
+  d.child_list = at(L.o_child_list);
+  d.tree = b->seg_parent ? 1 : 0;
   {
     size_t off = 0;
     auto take = [&](size_t n) { size_t o = off; off = align_up(off + n, 256); return o; };

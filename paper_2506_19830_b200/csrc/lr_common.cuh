@@ -17,6 +17,7 @@
 namespace lr {
 
 constexpr int kPage = 16;
+constexpr int kMaxTreeDepth = 8;  // deepest node of a draft-step tree (tree mode only; a chain may be longer)
 
 // Device status word layout: [0] = code (0 ok, 1 timeout, 2 bounds), [1] = detail.
 enum DevStatus : int { kDevOk = 0, kDevTimeout = 1, kDevBounds = 2 };
@@ -36,6 +37,13 @@ struct DevBatch {
   const int32_t *chain_tok;   // [n_span + n_req]
   const int32_t *tail_pg;     // [n_branch + n_req]
   const int32_t *compact_stage_off;  // [n_req+1] staging-token range of each request in lr_compact
+  // Tree of draft steps.  Spans are numbered in depth-first order per request (prefix 0); span c is seen
+  // from node n iff span_tin[c] <= span_tin[n] <= span_last[c] (last = highest number in c's subtree).  On the
+  // nested chain tin = c and last = gamma.  Children of span s: child_list[child_off[s] .. child_off[s+1]),
+  // local indices in increasing order.
+  const int32_t *span_tin, *span_last;  // [n_span]
+  const int32_t *child_off, *child_list;  // [n_span+1], [n_span]
+  int32_t tree;  // 1 when the batch gave seg_parent
   int32_t n_req, n_branch, n_span, n_page_slots, n_q_rows;
   int32_t n_q_heads, n_kv_heads, head_dim, group;
   int64_t n_pool_pages;
@@ -54,10 +62,10 @@ struct DevBatch {
 // contribute to a target each writes an fp32 partial and a second kernel merges.
 struct TcPage {      // one per extended-chain page
   int32_t page;      // physical page id
-  uint32_t meta;     // bits 0-4 valid tokens (0..16), 5-12 min depth to see it, 13-20 owner branch (local, +1; 0 = chain), 21-31 first tail token index of the page / 16
+  uint32_t meta;     // bits 0-4 valid tokens (0..16), 5-12 and 21-28 (chain pages) first and last depth-first node number that sees it, 13-20 owner branch (local, +1; 0 = chain), 21-31 (tail pages) first tail token index of the page / 16
 };
 struct TcRow {       // one per query row of the batch
-  int32_t depth_branch;  // depth | local branch index << 16
+  int32_t depth_branch;  // depth-first number of the branch's node | local branch index << 16
   int32_t limit;         // last tail token the row sees
 };
 struct TcPiece {
@@ -150,7 +158,9 @@ struct TcHostPlan {
   // scratch region behind the image: (exponent, sum) pairs, then fp32 partial outputs
   size_t s_ml = 0, s_o = 0, scratch_bytes = 0, scratch_zero_bytes = 0;
 };
-int tc_build_host_plan(const lr_ctx *ctx, const lr_batch *b, const int32_t *req_br_off, TcHostPlan &out, Image &img);
+// span_tin / span_last: depth-first interval labels of the spans ([n_span] each, see DevBatch)
+int tc_build_host_plan(const lr_ctx *ctx, const lr_batch *b, const int32_t *req_br_off, const int32_t *span_tin,
+                       const int32_t *span_last, TcHostPlan &out, Image &img);
 void tc_bind_device_plan(const TcHostPlan &h, unsigned char *image_base, unsigned char *scratch_base, lr_plan *p);
 
 void set_error(const char *fmt, ...);

@@ -90,6 +90,30 @@ def test_validation_rejects_each_broken_rule():
         assert e.value.status == -1, i
 
 
+def test_tree_batches_validate_and_broken_trees_are_rejected():
+    from lr_workloads import Model, build_batch, make_random_tree, make_tree
+    for seed in range(10):
+        w = make_random_tree(seed)
+        B.lr_validate_batch(w.batch.model, w.batch)
+    w = make_tree(2, 3, size="tiny", with_logits=False, with_kv=False)
+    b = w.batch
+    B.lr_validate_batch(b.model, b)
+    bad = [
+        _mut(b, "seg_parent", 1, 1),  # a segment that continues itself
+        _mut(b, "seg_parent", 2, 5),  # ... or a later segment
+        _mut(b, "seg_parent", 3, -1),
+    ]
+    # a chain of nine steps written as a tree is deeper than tree mode allows; as a plain chain it is fine
+    rng = np.random.default_rng(0)
+    req = {"P": 5, "segs": [3] * 9, "branches": [(9, 2, 2, 2)]}
+    B.lr_validate_batch(Model(2, 1, 64, 16), build_batch(Model(2, 1, 64, 16), [req], rng))
+    bad.append(build_batch(Model(2, 1, 64, 16), [dict(req, parents=list(range(9)))], rng))
+    for i, x in enumerate(bad):
+        with pytest.raises(B.LrError) as e:
+            B.lr_validate_batch(x.model, x)
+        assert e.value.status == -1, i
+
+
 def test_unsupported_geometry():
     w = make_random_small(2)
     import dataclasses
