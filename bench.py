@@ -59,12 +59,37 @@ def attention_work(batch):
     for b in range(batch.n_branch):
         r = int(batch.br_req[b])
         s0 = int(batch.req_span_off[r])
-        chain = int(batch.span_len[s0 : s0 + 1 + int(batch.br_depth[b])].sum())
+        if batch.seg_parent is None:
+            chain = int(batch.span_len[s0 : s0 + 1 + int(batch.br_depth[b])].sum())
+        else:  # tree of draft steps: the prefix and the steps between it and the branch's node
+            chain, node = int(batch.span_len[s0]), int(batch.br_depth[b])
+            while node != 0:
+                chain += int(batch.span_len[s0 + node])
+                node = int(batch.seg_parent[s0 + node])
         q_len = int(batch.cu_q[b + 1] - batch.cu_q[b])
         own = int(batch.br_own_len[b])
         vis += sum(chain + own - q_len + i + 1 for i in range(q_len))
     flops = 4 * m.n_q_heads * m.head_dim * vis
     return kv_bytes + qo_bytes, flops
+
+
+def make_workload(args, rank=None):
+    """The configuration the flags name; with a rank, that rank's independent batch (seed offset by rank)."""
+    from lr_workloads import make_config, make_tree
+
+    def seeded(seed):
+        if rank is None:
+            return seed
+        import paper_2506_19830_b200.sharding as S
+        return S.rank_seed(seed, rank)
+
+    if args.tree:
+        parts = args.tree.split(",")
+        W, gamma, size = int(parts[0]), int(parts[1]), (parts[2] if len(parts) > 2 else "layer")
+        w = make_tree(W, gamma, seed=seeded(20250700 + 16 * W + gamma), size=size)
+        return w, w.name
+    w = make_config(args.config, seed=seeded(20250619 + args.config), carry_in=args.carry_in)
+    return w, f"config{args.config}_{w.name}"
 
 
 def accept_bytes(batch):
@@ -152,9 +177,7 @@ def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return 0
-    from lr_workloads import make_config
-
-    w = make_config(args.config, carry_in=args.carry_in)
+    w, w_label = make_workload(args)
     tokens = w.batch.n_verified_tokens
     for _ in range(args.warmup):
         oracle_pass_seconds(w, 0.0, 1)
@@ -168,11 +191,11 @@ def run_reference(args):
     sec = sum(times) / len(times)
     cores = host_threads()
     val = tokens / sec
-    sample = f"whole pass of config {args.config} ({w.name}), one batch per step, {len(times)} steps"
+    sample = f"whole pass of {w_label}, one batch per step, {len(times)} steps"
     line = {
         "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": len(times),
         "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "f64", "data": "synthetic", "config": {"workload": f"config{args.config}_{w.name}", "seed": w.seed},
+        "dtype": "f64", "data": "synthetic", "config": {"workload": w_label, "seed": w.seed},
         "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -193,6 +216,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--carry-in", action="store_true", help="q_len = L + 1 per branch (the last accepted token is a query too)")
+    ap.add_argument("--tree", default="", help="W,GAMMA[,tiny|layer|serving]: multi-branch drafting workload instead of --config")
     ap.add_argument("--no-overlap", action="store_true", help="run the three steps of a pass strictly one after another")
     ap.add_argument("--no-graph", action="store_true", help="issue every launch from Python instead of replaying CUDA graphs")
     ap.add_argument("--path", type=int, default=0, help="attention path: 0 auto, 1 CUDA cores, 2 tensor cores")
@@ -203,7 +227,6 @@ def main():
     import torch
     import torch.distributed as dist
 
-    from lr_workloads import make_config
     from paper_2506_19830_b200 import binding as B
     from paper_2506_19830_b200 import runner as R
     from paper_2506_19830_b200 import sharding as S
@@ -218,7 +241,7 @@ def main():
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device(dev))
 
-    w = make_config(args.config, seed=S.rank_seed(20250619 + args.config, rank), carry_in=args.carry_in)
+    w, w_label = make_workload(args, rank)
     b, t = w.batch, w.tensors
     ctx = B.Context(b.model, local)
     plan = B.Plan(ctx, b)
@@ -418,7 +441,7 @@ def main():
         # dram__bytes_read.sum + dram__bytes_write.sum of one attn_tc_kernel launch on this workload (ncu
         # captures summarised under profiles/, taken on the kernels as they are); None where not captured
         traffic = ({2: 17_960_704 + 0, 3: 274_865_152 + 8_119_808}.get(args.config)
-                   if args.path == 0 and not args.carry_in else None)
+                   if args.path == 0 and not args.carry_in and not args.tree else None)
         roof.update({"traffic": traffic, "kernel": "lr_verify_attention", "kernel_us": kernel_us["attention"],
                      "algorithmic_bytes": a_bytes, "algorithmic_flops": a_flops, "peak_source": f"of {peak_kind}", "timed": "attn_tc_kernel + attn_tc_merge_kernel",
                      "roofline_us": max(hbm_time, tc_time) * 1e6})
@@ -451,12 +474,12 @@ def main():
         if not args.no_cpu_baseline:
             sec, n = oracle_pass_seconds(w, args.cpu_seconds)
             cpu = {"value": b.n_verified_tokens / sec, "unit": UNIT, "cores": host_threads(), "kind": "oracle",
-                   "sample": f"{n} whole passes of the same workload (config {args.config}), {sec * 1e3:.1f} ms each",
+                   "sample": f"{n} whole passes of the same workload ({w_label}), {sec * 1e3:.1f} ms each",
                    "ms_per_pass": sec * 1e3}
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W, "ms_per_step": ms_step,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": f"config{args.config}_{w.name}", "seed": w.seed, "requests_per_gpu": b.n_req,
+            "config": {"workload": w_label, "seed": w.seed, "requests_per_gpu": b.n_req,
                        "branches_per_gpu": b.n_branch, "kv_tokens_per_gpu": b.kv_tokens(), "verified_tokens_per_gpu": b.n_verified_tokens,
                        "l2_policy": f"rotating {copies} copies of KV pools and logits ({copies * per_copy / 1e6:.0f} MB > L2)",
                        "attention_path": args.path, "carry_in": bool(args.carry_in), "cuda_graph": bool(graphed), "overlap": "attention || (accept -> commit) on two streams" if overlap_stream is not None else "none",
