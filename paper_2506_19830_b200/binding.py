@@ -45,6 +45,10 @@ class lr_batch(C.Structure):
     ] + [("n_pool_pages", C.c_int64), ("seg_parent", _I32P)]
 
 
+class lr_cycle_stats(C.Structure):
+    _fields_ = [(n, C.c_int64) for n in ("stages", "steps", "time", "verdicts_used", "peak_in_flight")]
+
+
 class lr_pass_host_io(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in (
         "q_h", "logits_h", "draft_ids_h", "verdict_h", "out_h", "n_accept_h", "bonus_id_h", "n_steps_accepted_h",
@@ -79,6 +83,10 @@ def lib() -> C.CDLL:
             "lr_accept_sample_scratch_bytes": [vp, i32, C.POINTER(sz)],
             "lr_accept_sample": [vp, vp, i64, vp, vp, i32, i32, f32, vp, vp, vp, vp, vp, vp, vp],
             "lr_commit": [vp] + [vp] * 10 + [vp],
+            "lr_cycle_simulate_sync": [i32, i64, i64, vp, i64, C.POINTER(lr_cycle_stats)],
+            "lr_cycle_simulate_async": [i32, i64, i64, vp, i64, C.POINTER(lr_cycle_stats)],
+            "lr_cycle_best_strategy": [i32, C.c_double, C.c_double, C.c_double, C.c_double, i32, C.POINTER(i32),
+                                       C.POINTER(i32), C.POINTER(C.c_double)],
             "lr_compact_scratch_bytes": [vp, C.POINTER(sz)],
             "lr_compact": [vp] * 10,
             "lr_pass_staging_bytes": [vp, C.POINTER(sz)],
@@ -91,6 +99,8 @@ def lib() -> C.CDLL:
             fn.restype = C.c_int
         L.lr_launch_count.argtypes = [vp]
         L.lr_launch_count.restype = C.c_int64
+        L.lr_cycle_speedup.argtypes = [i32, i32, C.c_double, C.c_double]
+        L.lr_cycle_speedup.restype = C.c_double
         L.lr_strerror.argtypes = [C.c_int]
         L.lr_strerror.restype = C.c_char_p
         L.lr_last_error.argtypes = []
@@ -290,3 +300,33 @@ class Plan:
         _check(lib().lr_verify_pass_host(self.handle, C.byref(io), _ptr(k_pool), _ptr(v_pool), staging.data_ptr() + off,
                                          staging.numel() - off, float(softmax_scale), _stream_ptr(stream)),
                "lr_verify_pass_host")
+
+
+# ---- host-side cycle model (no device needed) --------------------------------------------------------
+def _stats(st: lr_cycle_stats) -> dict:
+    return {n: int(getattr(st, n)) for n, _ in lr_cycle_stats._fields_}
+
+
+def lr_cycle_simulate_sync(gamma: int, num: int, den: int, verdicts) -> dict:
+    v = np.ascontiguousarray(verdicts, dtype=np.uint8)
+    st = lr_cycle_stats()
+    _check(lib().lr_cycle_simulate_sync(gamma, num, den, v.ctypes.data, len(v), C.byref(st)), "lr_cycle_simulate_sync")
+    return _stats(st)
+
+
+def lr_cycle_simulate_async(gamma: int, num: int, den: int, verdicts) -> dict:
+    v = np.ascontiguousarray(verdicts, dtype=np.uint8)
+    st = lr_cycle_stats()
+    _check(lib().lr_cycle_simulate_async(gamma, num, den, v.ctypes.data, len(v), C.byref(st)), "lr_cycle_simulate_async")
+    return _stats(st)
+
+
+def lr_cycle_speedup(mode: int, k: int, alpha: float, c: float) -> float:
+    return float(lib().lr_cycle_speedup(mode, k, alpha, c))
+
+
+def lr_cycle_best_strategy(budget: int, alpha1: float, c1: float, alpha2: float, c2: float, asynchronous: bool = True):
+    k1, k2, h = C.c_int32(), C.c_int32(), C.c_double()
+    _check(lib().lr_cycle_best_strategy(budget, alpha1, c1, alpha2, c2, int(asynchronous), C.byref(k1), C.byref(k2),
+                                        C.byref(h)), "lr_cycle_best_strategy")
+    return k1.value, k2.value, h.value
