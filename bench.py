@@ -246,6 +246,15 @@ def main():
     ctx = B.Context(b.model, local)
     plan = B.Plan(ctx, b)
     plan.lr_plan_set_attention_path(args.path)
+    # host cost of planning a batch (a serving loop plans once per cycle: the structure changes every time)
+    t_plan = []
+    for _ in range(5):
+        t0 = time.perf_counter()
+        tmp = B.Plan(ctx, b)
+        torch.cuda.synchronize()
+        t_plan.append(time.perf_counter() - t0)
+        tmp.close()
+    plan_ms = 1e3 * float(np.median(t_plan))
     x0 = R.DeviceInputs(b, t, dev)
     y = R.PassOutputs(b, dev)
     per_copy = 2 * x0.k_pool.numel() * 2 + x0.logits.numel() * 2
@@ -486,6 +495,7 @@ def main():
                        "per_kernel_timing": "K back-to-back launches of the kernel alone over the rotating copies"},
             "roofline": roof, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
             "kernels": kernels,
+            "plan_create_host_ms": plan_ms,
         }
         print(json.dumps(line))
     if world > 1:

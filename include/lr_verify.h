@@ -138,6 +138,9 @@ int lr_plan_bytes(const lr_ctx *ctx, const lr_batch *batch_h, size_t *bytes_out)
  * the same plan must not overlap on the device (they share the workspace). */
 int lr_plan_create(lr_ctx *ctx, const lr_batch *batch_h, void *workspace_d, size_t workspace_bytes,
                    void *stream, lr_plan **out);
+/* Releases the plan (not the workspace, which is the caller's).  The plan's pinned host buffer goes back to its
+ * context for the next plan, so destroy every plan before its context.  Contexts and their plans are not
+ * thread-safe: one thread at a time per context. */
 int lr_plan_destroy(lr_plan *plan);
 
 /* ---- the three steps ---------------------------------------------------- */

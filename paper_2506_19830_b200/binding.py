@@ -9,6 +9,7 @@ from __future__ import annotations
 
 import ctypes as C
 import os
+import weakref
 from typing import Optional
 
 import numpy as np
@@ -170,9 +171,12 @@ class Context:
         m = _model_struct(model)
         _check(lib().lr_create(C.byref(h), C.byref(m), device), "lr_create")
         self.handle = h
+        self._plans = weakref.WeakSet()  # plans must be destroyed before their context
 
     def close(self):
         if self.handle:
+            for p in list(self._plans):
+                p.close()
             lib().lr_destroy(self.handle)
             self.handle = None
 
@@ -243,6 +247,7 @@ class Plan:
         _check(lib().lr_plan_create(ctx.handle, C.byref(self.host.c), self._ws_ptr, n.value, _stream_ptr(stream), C.byref(h)),
                "lr_plan_create")
         self.handle = h
+        ctx._plans.add(self)
         self.n_req = self.host.c.n_req
         self.n_branch = self.host.c.n_branch
         self.n_page_slots = self.host.c.n_page_slots

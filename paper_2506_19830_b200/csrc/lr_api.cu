@@ -283,8 +283,49 @@ extern "C" int lr_create(lr_ctx **out, const lr_model *m, int device) {
 }
 
 extern "C" int lr_destroy(lr_ctx *ctx) {
+  if (ctx) {
+    for (auto &pb : ctx->pinned_free) {
+      cudaEventSynchronize(pb.uploaded);
+      cudaEventDestroy(pb.uploaded);
+      cudaFreeHost(pb.ptr);
+    }
+  }
   delete ctx;
   return LR_OK;
+}
+
+// A pinned buffer of at least `bytes`: the smallest cached one that fits, else a new one (capacity rounded up to a
+// power of two, at least 64 KB, so that the next plan of a similar batch fits too).
+static int take_pinned(lr_ctx *ctx, size_t bytes, void **ptr, size_t *cap, cudaEvent_t *ev) {
+  int best = -1;
+  for (int i = 0; i < (int)ctx->pinned_free.size(); ++i)
+    if (ctx->pinned_free[i].cap >= bytes && (best < 0 || ctx->pinned_free[i].cap < ctx->pinned_free[best].cap)) best = i;
+  if (best >= 0) {
+    lr_ctx::PinnedBuf pb = ctx->pinned_free[best];
+    ctx->pinned_free.erase(ctx->pinned_free.begin() + best);
+    if (int rc = cuda_fail(cudaEventSynchronize(pb.uploaded), "cudaEventSynchronize(pinned buffer)")) return rc;
+    *ptr = pb.ptr; *cap = pb.cap; *ev = pb.uploaded;
+    return LR_OK;
+  }
+  size_t c = 64 << 10;
+  while (c < bytes) c <<= 1;
+  if (int rc = cuda_fail(cudaMallocHost(ptr, c), "cudaMallocHost(plan image)")) return rc;
+  if (int rc = cuda_fail(cudaEventCreateWithFlags(ev, cudaEventDisableTiming), "cudaEventCreate")) {
+    cudaFreeHost(*ptr);
+    return rc;
+  }
+  *cap = c;
+  return LR_OK;
+}
+
+static void give_back_pinned(lr_ctx *ctx, void *ptr, size_t cap, cudaEvent_t ev) {
+  if (ctx->pinned_free.size() < 8) {
+    ctx->pinned_free.push_back({ptr, cap, ev});
+    return;
+  }
+  cudaEventSynchronize(ev);
+  cudaEventDestroy(ev);
+  cudaFreeHost(ptr);
 }
 
 extern "C" int64_t lr_launch_count(const lr_ctx *ctx) { return ctx ? ctx->launches : 0; }
@@ -326,7 +367,7 @@ extern "C" int lr_plan_create(lr_ctx *ctx, const lr_batch *b, void *ws, size_t w
   p->workspace_d = ws;
   p->workspace_bytes = ws_bytes;
   p->attention_path = 0;
-  if (int rc = cuda_fail(cudaMallocHost(&p->pinned, L.image_bytes), "cudaMallocHost(plan image)")) {
+  if (int rc = take_pinned(ctx, L.image_bytes, &p->pinned, &p->pinned_cap, &p->uploaded)) {
     delete p;
     return rc;
   }
@@ -386,8 +427,9 @@ extern "C" int lr_plan_create(lr_ctx *ctx, const lr_batch *b, void *ws, size_t w
   cudaError_t e = cudaMemcpyAsync(ws, p->pinned, L.image_bytes, cudaMemcpyHostToDevice, s);
   if (e == cudaSuccess && L.tc.scratch_zero_bytes)
     e = cudaMemsetAsync(base + L.image_bytes, 0, L.tc.scratch_zero_bytes, s);
+  if (e == cudaSuccess) e = cudaEventRecord(p->uploaded, s);
   if (e != cudaSuccess) {
-    cudaFreeHost(p->pinned);
+    give_back_pinned(ctx, p->pinned, p->pinned_cap, p->uploaded);
     delete p;
     return cuda_fail(e, "plan upload");
   }
@@ -397,7 +439,7 @@ extern "C" int lr_plan_create(lr_ctx *ctx, const lr_batch *b, void *ws, size_t w
 
 extern "C" int lr_plan_destroy(lr_plan *p) {
   if (!p) return LR_OK;
-  if (p->pinned) cudaFreeHost(p->pinned);
+  if (p->pinned) give_back_pinned(p->ctx, p->pinned, p->pinned_cap, p->uploaded);
   delete p;
   return LR_OK;
 }

@@ -118,6 +118,10 @@ struct lr_ctx {
   void *tmap_encode;  // cuTensorMapEncodeTiled entry point (driver), resolved lazily
   struct TmapEntry { const void *ptr; int64_t n; int kind; alignas(64) unsigned char map[128]; };
   std::vector<TmapEntry> tmaps;
+  // Pinned host buffers of destroyed plans, kept for the next plan: allocating and freeing pinned memory costs
+  // far more than building a plan.  `uploaded` is recorded after the buffer's last upload; a new user waits on it.
+  struct PinnedBuf { void *ptr; size_t cap; cudaEvent_t uploaded; };
+  std::vector<PinnedBuf> pinned_free;
 };
 
 struct lr_plan {
@@ -128,6 +132,8 @@ struct lr_plan {
   int attention_path;     // 0 auto, 1 generic, 2 tensor core
   std::vector<unsigned char> staging;  // host copy of the uploaded image (kept alive for the async copy)
   void *pinned;           // pinned host image
+  size_t pinned_cap;
+  cudaEvent_t uploaded;   // recorded after the image's upload
   size_t image_bytes;
   void *workspace_d;
   size_t workspace_bytes;
