@@ -24,9 +24,15 @@
 // softmax warpgroups with setmaxnreg):
 //   warp 8      TMA producer: the Q tiles of a piece (3-D boxes: 64 channels x G
 //               heads x T tokens, so that the rows land packed) and, per tile,
-//               16 + 16 bulk tensor copies (one per page and 64-channel half, K
-//               and V) into a 5-stage ring of 32 KB buffers, all in the
-//               128-byte-swizzled layout the MMA descriptors read.  No multicast.
+//               8 + 8 bulk tensor copies (one 4 KB box per page, K and V) into a
+//               5-stage ring of 32 KB buffers.  A box is a 4-D view of the page,
+//               [8-key group][channel half][8 keys][64 channels], so a tile lies in
+//               shared memory as 1024-byte swizzle atoms, the two channel halves of
+//               an 8-key group side by side (groups 2048 bytes apart): the layout
+//               the MMA descriptors read with SBO = 2048.  One box per page rather
+//               than one per page half matters: the producer spends about 100
+//               cycles per box, and 32 boxes per tile made it a bottleneck.
+//               No multicast.
 //   warps 9, 10 MMA issuers of stream 0 and 1 (warp 11 idles): tcgen05.mma (M=128, N=128, K=16,
 //               bf16 -> fp32) for S = Q K^T (both operands in shared memory) and
 //               O += P V (P read from tensor memory, V from shared memory as the
@@ -69,6 +75,8 @@ constexpr int kD = 128;
 constexpr int kStages = 5;
 constexpr int kTileBytes = 32768;  // [2 halves of 64 channels][128 keys or rows][128 B]
 constexpr int kHalfBytes = 16384;
+constexpr int kAtomBytes = 1024;   // K/V tiles: 8 keys x 64 channels, one 128-byte-swizzle atom
+constexpr int kGroupBytes = 2048;  // ... two atoms (the two channel halves) per 8-key group
 constexpr int kThreads = 384;
 constexpr int kPagesPerTile = 8;
 constexpr uint64_t kWaitLimitNs = 1000ull * 1000ull * 1000ull;  // one second per wait, measured on the global timer
@@ -132,10 +140,10 @@ __device__ __forceinline__ void tc_commit(uint64_t *bar) {
 }
 
 // Tiled bulk tensor copies global -> shared, completion on an mbarrier (no multicast).
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int32_t x, int32_t y, uint64_t *bar) {
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *map, int32_t x, int32_t y, int32_t z, int32_t w, uint64_t *bar) {
   asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(dst),
-      "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y)
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];" ::"r"(dst),
+      "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y), "r"(z), "r"(w)
       : "memory");
 }
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, int32_t x, int32_t y, int32_t z, uint64_t *bar) {
@@ -490,16 +498,16 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant_
           pg_cur = pg_nxt;
           pg_nxt = load_chunk(c_cur + 1);
         }
-        const int32_t page = __shfl_sync(0xFFFFFFFFu, (t >> 2) == c_cur ? pg_cur : pg_nxt, (t & 3) * 8 + ((lane & 15) >> 1));
+        const int32_t page = __shfl_sync(0xFFFFFFFFu, (t >> 2) == c_cur ? pg_cur : pg_nxt, (t & 3) * 8 + (lane & 7));
         const int npages = min(kPagesPerTile, rq.n_pages - t * kPagesPerTile);
         const uint32_t stage = ring % kStages;
         ok = wait_bar(&ctrl->kv_empty[stage], ((ring / kStages) & 1u) ^ 1u, ctrl, d.status, 210);
         if (!ok) break;
         if (lane == 0) mbar_arrive_expect_tx(&ctrl->kv_full[stage], (uint32_t)npages * 4096u);
         __syncwarp();
-        if (lane < 16 && page >= 0) {
-          const uint32_t dst = smem_u32(kv_smem + stage * kTileBytes) + (lane & 1) * kHalfBytes + (lane >> 1) * 2048;
-          tma_load_2d(dst, is_v ? &v_map : &k_map, (lane & 1) * 64, (int32_t)(((int64_t)page * d.n_kv_heads + pi.kv_head) * kPage),
+        if (lane < 8 && page >= 0) {  // one 4 KB box per page: two 8-key groups x two d halves
+          const uint32_t dst = smem_u32(kv_smem + stage * kTileBytes) + lane * 4096;
+          tma_load_4d(dst, is_v ? &v_map : &k_map, 0, 0, 0, (int32_t)(((int64_t)page * d.n_kv_heads + pi.kv_head) * 2),
                       &ctrl->kv_full[stage]);
         }
       }
@@ -525,23 +533,23 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant_
     const uint32_t q_addr = smem_u32(q_smem), kv_addr = smem_u32(kv_smem);
     const uint32_t s_tmem = tmem + s * 128, o_tmem = tmem + 256 + s * 128;
     // Descriptors differ from a base only in the start-address field (units of 16 bytes).
-    const uint64_t qdesc0 = make_desc(q_addr, 16, 1024), kdesc0 = make_desc(kv_addr, 16, 1024),
-                   vdesc0 = make_desc(kv_addr, kHalfBytes, 1024);
+    const uint64_t qdesc0 = make_desc(q_addr, 16, 1024), kdesc0 = make_desc(kv_addr, 16, kGroupBytes),
+                   vdesc0 = make_desc(kv_addr, kAtomBytes, kGroupBytes);
     auto issue_qk = [&](int m, uint32_t stage, int half) {  // S_s[half] = Q_m K^T over 64 of the 128 keys
       const uint64_t a = qdesc0 + (uint64_t)(m * (kTileBytes >> 4)),
-                     b = kdesc0 + (uint64_t)(stage * (kTileBytes >> 4) + half * (64 * 128 >> 4));
+                     b = kdesc0 + (uint64_t)(stage * (kTileBytes >> 4) + half * (8 * kGroupBytes >> 4));
 #pragma unroll
       for (int h = 0; h < 2; ++h)
 #pragma unroll
         for (int kk = 0; kk < 4; ++kk)
-          mma_ss(s_tmem + half * 64, a + (uint64_t)(h * (kHalfBytes >> 4) + kk * 2), b + (uint64_t)(h * (kHalfBytes >> 4) + kk * 2),
+          mma_ss(s_tmem + half * 64, a + (uint64_t)(h * (kHalfBytes >> 4) + kk * 2), b + (uint64_t)(h * (kAtomBytes >> 4) + kk * 2),
                  kIdescQK, (h | kk) != 0);
     };
     auto issue_pv = [&](uint32_t stage, int half, bool acc) {  // O_s (+)= P_s[half] V over 64 of the 128 keys
-      const uint64_t b = vdesc0 + (uint64_t)(stage * (kTileBytes >> 4) + half * (4 * 2048 >> 4));
+      const uint64_t b = vdesc0 + (uint64_t)(stage * (kTileBytes >> 4) + half * (8 * kGroupBytes >> 4));
 #pragma unroll
       for (int k4 = 0; k4 < 4; ++k4)
-        mma_ts(o_tmem, s_tmem + half * 64 + k4 * 8, b + (uint64_t)(k4 * (2048 >> 4)), kIdescPV, acc || k4 != 0);
+        mma_ts(o_tmem, s_tmem + half * 64 + k4 * 8, b + (uint64_t)(k4 * (2 * kGroupBytes >> 4)), kIdescPV, acc || k4 != 0);
     };
     for (int pc = piece0; pc < piece1 && ok; ++pc, ++pc_idx) {
       const TcPiece pi = pc == piece0 ? head->first : tc.pieces[pc];
@@ -595,7 +603,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant_
             const int valid = pg[p].meta & 31;
             for (int idx = lane; idx < (kPage - valid) * 16; idx += 32) {
               const int key = p * kPage + valid + (idx >> 4), h = (idx >> 3) & 1, ch = idx & 7;
-              *reinterpret_cast<uint4 *>(vs + h * kHalfBytes + key * 128 + ch * 16) = make_uint4(0, 0, 0, 0);
+              *reinterpret_cast<uint4 *>(vs + (key >> 3) * kGroupBytes + h * kAtomBytes + (key & 7) * 128 + ch * 16) = make_uint4(0, 0, 0, 0);
             }
           }
           fence_proxy_async();
@@ -886,7 +894,8 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t
                                   const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-// kind 0: a KV pool of n pages as [pages * kv heads * 16][128], box = one page half (16 rows x 64 channels)
+// kind 0: a KV pool of n pages viewed as [8-key groups][2 channel halves][8 keys][64 channels]; box = one page of one
+//         KV head (4 KB), which lands in shared memory as two 8-key groups of two 1024-byte swizzle atoms each
 // kind 1: Q of n rows as [rows][q heads][128], box = 64 channels x G heads x T tokens
 int get_map(lr_ctx *ctx, int kind, const void *ptr, int64_t n, const CUtensorMap **out) {
   for (auto &e : ctx->tmaps)
@@ -913,12 +922,13 @@ int get_map(lr_ctx *ctx, int kind, const void *ptr, int64_t n, const CUtensorMap
   const lr_model &m = ctx->model;
   CUresult r;
   if (kind == 0) {
-    cuuint64_t dims[2] = {(cuuint64_t)kD, (cuuint64_t)n * m.n_kv_heads * kPage};
-    cuuint64_t strides[1] = {(cuuint64_t)kD * 2};
-    cuuint32_t box[2] = {64, kPage};
-    cuuint32_t estr[2] = {1, 1};
+    // [8-key group][channel half][key in group][64 channels]: one box = one page of one KV head (4 KB)
+    cuuint64_t dims[4] = {64, 8, 2, (cuuint64_t)n * m.n_kv_heads * (kPage / 8)};
+    cuuint64_t strides[3] = {(cuuint64_t)kD * 2, 128, (cuuint64_t)kD * 2 * 8};
+    cuuint32_t box[4] = {64, 8, 2, kPage / 8};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
     r = reinterpret_cast<EncodeTiledFn>(ctx->tmap_encode)(
-        reinterpret_cast<CUtensorMap *>(ent.map), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(ptr), dims, strides, box,
+        reinterpret_cast<CUtensorMap *>(ent.map), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(ptr), dims, strides, box,
         estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   } else {
