@@ -128,6 +128,19 @@ __device__ __forceinline__ uint32_t mbar_test_wait(uint64_t *bar, uint32_t parit
       : "memory");
   return ok;
 }
+// both tests in flight together: bit 0 = first barrier's phase complete, bit 1 = second's
+__device__ __forceinline__ uint32_t mbar_test_wait2(uint64_t *bar_a, uint32_t parity_a, uint64_t *bar_b, uint32_t parity_b) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t.reg .b32 a, b;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 q, [%3], %4;\n\t"
+      "selp.b32 a, 1, 0, p;\n\tselp.b32 b, 2, 0, q;\n\tor.b32 %0, a, b;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar_a)), "r"(parity_a), "r"(smem_u32(bar_b)), "r"(parity_b)
+      : "memory");
+  return ok;
+}
 __device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -592,6 +605,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant_
       for (int j = 0; j < my_units && ok; ++j) {
         const int t = mode == 2 ? j : 2 * j + s;
         const uint32_t pos_v = ring_base + ord.pos_v(t), sV = pos_v % kStages;
+        if (mode == 2 && j + 1 < my_units && waited == pos_v &&
+            mbar_test_wait2(&ctrl->kv_full[pos_v % kStages], (pos_v / kStages) & 1u, &ctrl->kv_full[(pos_v + 1) % kStages],
+                            ((pos_v + 1) / kStages) & 1u) == 3u)
+          waited = pos_v + 2;  // V of this tile and K of the next (the position right behind it) have both landed
         ok = need(pos_v, 222);
         if (!ok) break;
         if (pi.tile_begin + t >= rq.n_dense_tiles) {
