@@ -976,6 +976,9 @@ int init_attn_tc_kernel() {
 }
 
 // ---- host planning -----------------------------------------------------------------
+// most CTAs worth using for a number of tiles (tiny problems: not one CTA per tile, their partial results cost more than they save)
+static int64_t kCtaPerTiles(int64_t tiles) { return tiles >= 64 ? tiles : tiles / 2; }
+
 int tc_build_host_plan(const lr_ctx *ctx, const lr_batch *b, const int32_t *req_br_off, const int32_t *span_tin,
                        const int32_t *span_last, TcHostPlan &out, Image &img) {
   out = TcHostPlan();
@@ -1041,45 +1044,66 @@ int tc_build_host_plan(const lr_ctx *ctx, const lr_batch *b, const int32_t *req_
       }
   }
   if (grps.empty()) return LR_OK;
-  // Cut the weighted tile sequence into n_cta contiguous ranges of equal weight: a tile belongs to the
-  // CTA whose weight interval [total*c/n, total*(c+1)/n) holds the tile's start position.
-  // The start of a group inside a CTA's range (epilogue, Q reload, pipeline ramp) is charged like
-  // kPieceStartTiles tiles, so such a CTA gets fewer tiles.
-  constexpr int kPieceStartTiles = 3;
-  int64_t total_w = 0, total_tiles = 0;
+  // Contiguous partition of the tile sequence (groups in order, tiles in order) over at most max_cta CTAs that
+  // minimises the largest CTA load.  A tile costs its group's weight; every piece -- a CTA's share of one group --
+  // costs kPieceStartTiles tiles more (Q load, pipeline ramp, epilogue), so a CTA that spans a group boundary gets
+  // fewer tiles; a tile that needs masks (anything past the full prefix pages) costs 8/5 of a dense one (measured).  For a load limit L the greedy fill (a CTA takes tiles while it stays within L) needs the fewest
+  // CTAs possible; the smallest feasible L is found by bisection.  At most one CTA per two tiles: smaller shares
+  // only add partial results to merge.
+  constexpr int kPieceStartTiles = 3, kDense = 5, kMasked = 8;  // costs in fifths of a dense tile
+  auto tile_cost = [&](const Grp &g, int t) -> int64_t {
+    return (int64_t)g.weight * (t >= reqs[g.req].n_dense_tiles ? kMasked : kDense);
+  };
+  int64_t total_w = 0, total_tiles = 0, lo = 0;
   for (const Grp &g : grps) {
-    total_w += (int64_t)(g.n_tiles + kPieceStartTiles) * g.weight;
+    total_w += (int64_t)kPieceStartTiles * kDense * g.weight;
+    for (int t = 0; t < g.n_tiles; ++t) total_w += tile_cost(g, t);
     total_tiles += g.n_tiles;
+    lo = std::max<int64_t>(lo, (int64_t)(kPieceStartTiles * kDense + kMasked) * g.weight);
   }
-  const int n_cta = (int)std::min<int64_t>(ctx->sm_count, std::max<int64_t>(1, total_tiles / 2));
+  const int64_t max_cta = std::min<int64_t>(ctx->sm_count, std::max<int64_t>(1, kCtaPerTiles(total_tiles)));
+  // walks the partition for limit L; with `emit` it also records the pieces
   std::vector<TcPiece> pieces;
-  std::vector<int32_t> cta_off((size_t)n_cta + 1, 0);
-  std::vector<int> piece_group;
-  int64_t w_pos = 0;
-  int cta = 0, last_cta = -1;
-  for (size_t gi = 0; gi < grps.size(); ++gi) {
-    Grp &g = grps[gi];
-    g.first_piece = (int)pieces.size();
-    w_pos += (int64_t)kPieceStartTiles * g.weight;
-    for (int t = 0; t < g.n_tiles; ++t, w_pos += g.weight) {
-      while (cta + 1 < n_cta && w_pos >= total_w * (cta + 1) / n_cta) {
-        ++cta;
-        cta_off[cta] = (int32_t)pieces.size();
+  std::vector<int32_t> cta_off;
+  auto walk = [&](int64_t L, bool emit) -> int64_t {
+    int64_t n = 0, load = 0;
+    for (size_t gi = 0; gi < grps.size(); ++gi) {
+      Grp &g = grps[gi];
+      if (emit) g.first_piece = (int)pieces.size();
+      bool new_piece = true;
+      for (int t = 0; t < g.n_tiles; ++t) {
+        int64_t cost = tile_cost(g, t) + (new_piece ? (int64_t)kPieceStartTiles * kDense * g.weight : 0);
+        if (n == 0 || load + cost > L) {  // open the next CTA: its share of this group is a new piece
+          ++n;
+          load = 0;
+          new_piece = true;
+          cost = tile_cost(g, t) + (int64_t)kPieceStartTiles * kDense * g.weight;
+          if (emit) cta_off.push_back((int32_t)pieces.size());
+        }
+        load += cost;
+        if (emit) {
+          if (new_piece) {
+            TcPiece p;
+            p.req = g.req; p.kv_head = g.kv; p.mtile0 = g.mtile0; p.n_mt = g.n_mt; p.tile_begin = t; p.tile_end = t + 1;
+            p.slot[0] = p.slot[1] = -2;
+            pieces.push_back(p);
+          } else {
+            pieces.back().tile_end = t + 1;
+          }
+        }
+        new_piece = false;
       }
-      if (!pieces.empty() && piece_group.back() == (int)gi && last_cta == cta) {
-        pieces.back().tile_end = t + 1;  // same group, same CTA: extend the piece
-      } else {
-        TcPiece p;
-        p.req = g.req; p.kv_head = g.kv; p.mtile0 = g.mtile0; p.n_mt = g.n_mt; p.tile_begin = t; p.tile_end = t + 1;
-        p.slot[0] = p.slot[1] = -2;
-        pieces.push_back(p);
-        piece_group.push_back((int)gi);
-        last_cta = cta;
-      }
+      if (emit) g.n_pieces = (int)pieces.size() - g.first_piece;
     }
-    g.n_pieces = (int)pieces.size() - g.first_piece;
+    return n;
+  };
+  int64_t hi = total_w;  // one CTA takes everything
+  while (lo < hi) {
+    const int64_t mid = lo + (hi - lo) / 2;
+    if (walk(mid, false) <= max_cta) hi = mid; else lo = mid + 1;
   }
-  for (int c = cta + 1; c <= n_cta; ++c) cta_off[c] = (int32_t)pieces.size();
+  const int n_cta = (int)walk(lo, true);
+  cta_off.push_back((int32_t)pieces.size());
   // Targets (one M-tile of one group) and the streams that contribute to them, in piece order.
   int n_slots = 0;
   std::vector<TcTarget> targets;
