@@ -1062,7 +1062,8 @@ int tc_build_host_plan(const lr_ctx *ctx, const lr_batch *b, const int32_t *req_
     lo = std::max<int64_t>(lo, (int64_t)(kPieceStartTiles * kDense + kMasked) * g.weight);
   }
   const int64_t max_cta = std::min<int64_t>(ctx->sm_count, std::max<int64_t>(1, kCtaPerTiles(total_tiles)));
-  // walks the partition for limit L; with `emit` it also records the pieces
+  // walks the partition for limit L; with `emit` it also records the pieces.  A group is a run of dense tiles
+  // followed by a run of masked ones, each of uniform cost, so a walk takes O(CTAs + groups) steps.
   std::vector<TcPiece> pieces;
   std::vector<int32_t> cta_off;
   auto walk = [&](int64_t L, bool emit) -> int64_t {
@@ -1070,28 +1071,34 @@ int tc_build_host_plan(const lr_ctx *ctx, const lr_batch *b, const int32_t *req_
     for (size_t gi = 0; gi < grps.size(); ++gi) {
       Grp &g = grps[gi];
       if (emit) g.first_piece = (int)pieces.size();
+      const int64_t start = (int64_t)kPieceStartTiles * kDense * g.weight;
+      const int n_dense = std::min(g.n_tiles, reqs[g.req].n_dense_tiles);
       bool new_piece = true;
-      for (int t = 0; t < g.n_tiles; ++t) {
-        int64_t cost = tile_cost(g, t) + (new_piece ? (int64_t)kPieceStartTiles * kDense * g.weight : 0);
-        if (n == 0 || load + cost > L) {  // open the next CTA: its share of this group is a new piece
+      int t = 0;
+      while (t < g.n_tiles) {
+        const int run_end = t < n_dense ? n_dense : g.n_tiles;
+        const int64_t cost = tile_cost(g, t);
+        if (n == 0 || load + cost + (new_piece ? start : 0) > L) {  // open the next CTA: its share of this group is a new piece
           ++n;
           load = 0;
           new_piece = true;
-          cost = tile_cost(g, t) + (int64_t)kPieceStartTiles * kDense * g.weight;
           if (emit) cta_off.push_back((int32_t)pieces.size());
         }
-        load += cost;
+        if (new_piece) load += start;
+        const int k = (int)std::max<int64_t>(1, std::min<int64_t>(run_end - t, (L - load) / cost));
+        load += (int64_t)k * cost;
         if (emit) {
           if (new_piece) {
             TcPiece p;
-            p.req = g.req; p.kv_head = g.kv; p.mtile0 = g.mtile0; p.n_mt = g.n_mt; p.tile_begin = t; p.tile_end = t + 1;
+            p.req = g.req; p.kv_head = g.kv; p.mtile0 = g.mtile0; p.n_mt = g.n_mt; p.tile_begin = t; p.tile_end = t + k;
             p.slot[0] = p.slot[1] = -2;
             pieces.push_back(p);
           } else {
-            pieces.back().tile_end = t + 1;
+            pieces.back().tile_end = t + k;
           }
         }
         new_piece = false;
+        t += k;
       }
       if (emit) g.n_pieces = (int)pieces.size() - g.first_piece;
     }
