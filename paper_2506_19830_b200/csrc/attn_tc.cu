@@ -18,7 +18,9 @@
 // other.  A stream whose result is the only contribution to its M-tile writes
 // bf16 output; otherwise it writes an fp32 partial (reference exponent, sum,
 // unnormalised O) and a small second kernel merges the partials of an M-tile in
-// a fixed order.
+// a fixed order.  The two streams of a one-M-tile piece hold partial results of the
+// same rows; they are combined inside the CTA (stream 0 reads stream 1's accumulator
+// from tensor memory) and leave as one result.
 //
 // One CTA = 12 warps in three warpgroups (registers are moved from the service warps to the
 // softmax warpgroups with setmaxnreg):
@@ -89,10 +91,15 @@ struct __align__(8) Ctrl {
   uint64_t q_full, q_empty;
   uint64_t s_full[2][2], p_full[2][2], o_done[2];  // [stream][half]
   uint64_t epi_done, drain[2];
+  uint64_t xch;           // stream 1 -> stream 0: its (m, l) are published and its accumulator is final
   uint32_t tmem_base;
   int abort_flag;
+  float2 ml_xch[128];     // (reference exponent, row sum) of stream 1's rows, for the in-CTA combination
 };
-constexpr int kSmemBytes = 2 * kTileBytes + kStages * kTileBytes + 1024;  // tiles, then Ctrl; the base must be 1024-aligned
+constexpr int kCtrlBytes = 2048;
+static_assert(sizeof(Ctrl) <= kCtrlBytes, "Ctrl must fit behind the tiles");
+constexpr int kSmemBytes = 2 * kTileBytes + kStages * kTileBytes + kCtrlBytes;  // tiles, then Ctrl; the base must be 1024-aligned
+static_assert(kSmemBytes <= 227 * 1024, "shared memory per CTA");
 
 // ---- PTX wrappers ----------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -395,6 +402,71 @@ __device__ __forceinline__ float exp_half_max(const uint32_t (&v)[64], uint32_t 
   return acc0.x + acc0.y;
 }
 
+// The store epilogue of a softmax thread: row r of the accumulator at o_addr (and, when the CTA's two streams worked on
+// the same rows, of the other stream's at o_other, weighted) goes out as bf16 (slot < 0) or as an fp32 partial.
+// Not inlined: its two 64-register row buffers must not weigh on the register allocation of the sweep.
+__device__ __noinline__ void store_rows(uint32_t o_addr, uint32_t o_other, int slot, bool pair, float w_self, float w_other, float m_out,
+                                        float l_out, int r, int64_t q_index, uint16_t *__restrict__ out, float *__restrict__ lse,
+                                        float *__restrict__ partial_o, float *__restrict__ partial_ml) {
+          const bool any_other = pair && __any_sync(0xFFFFFFFFu, w_other > 0.f);
+          if (slot < 0) {
+            const float inv = 1.0f / l_out, a = w_self * inv, b = w_other * inv;
+#pragma unroll
+            for (int hf = 0; hf < 2; ++hf) {
+              uint32_t o[64];
+              tmem_ld64(o_addr + hf * 64, o);
+              tc_wait_ld();
+#pragma unroll
+              for (int c = 0; c < 64; ++c) o[c] = __float_as_uint(bits_f(o[c]) * a);
+              if (any_other) {  // the loads are warp-wide; a row whose other stream saw nothing keeps its own values
+                uint32_t p[64];
+                tmem_ld64(o_other + hf * 64, p);
+                tc_wait_ld();
+                if (w_other > 0.f) {
+#pragma unroll
+                  for (int c = 0; c < 64; ++c) o[c] = __float_as_uint(fmaf(bits_f(p[c]), b, bits_f(o[c])));
+                }
+              }
+              if (q_index >= 0) {
+                uint4 *dst = reinterpret_cast<uint4 *>(out + q_index * kD + hf * 64);
+#pragma unroll
+                for (int jj = 0; jj < 8; ++jj)
+                  dst[jj] = make_uint4(pack_bf16(bits_f(o[8 * jj]), bits_f(o[8 * jj + 1])), pack_bf16(bits_f(o[8 * jj + 2]), bits_f(o[8 * jj + 3])),
+                                       pack_bf16(bits_f(o[8 * jj + 4]), bits_f(o[8 * jj + 5])), pack_bf16(bits_f(o[8 * jj + 6]), bits_f(o[8 * jj + 7])));
+              }
+            }
+            if (lse != nullptr && q_index >= 0) lse[q_index] = (m_out + log2f(l_out)) * 0.6931471805599453f;
+          } else {
+            const int64_t prow = (int64_t)slot * 128 + r;
+#pragma unroll
+            for (int hf = 0; hf < 2; ++hf) {
+              uint32_t o[64];
+              tmem_ld64(o_addr + hf * 64, o);
+              tc_wait_ld();
+              if (pair) {
+#pragma unroll
+                for (int c = 0; c < 64; ++c) o[c] = __float_as_uint(bits_f(o[c]) * w_self);
+                if (any_other) {
+                  uint32_t p[64];
+                  tmem_ld64(o_other + hf * 64, p);
+                  tc_wait_ld();
+                  if (w_other > 0.f) {
+#pragma unroll
+                    for (int c = 0; c < 64; ++c) o[c] = __float_as_uint(fmaf(bits_f(p[c]), w_other, bits_f(o[c])));
+                  }
+                }
+              }
+              if (q_index >= 0) {
+                // chunk-major: 16-byte chunk k of row r at [slot][k][r], so a warp's store is 512 contiguous bytes
+                uint4 *dst = reinterpret_cast<uint4 *>(partial_o) + ((int64_t)slot * 32 + hf * 16) * 128 + r;
+#pragma unroll
+                for (int jj = 0; jj < 16; ++jj) dst[jj * 128] = make_uint4(o[4 * jj], o[4 * jj + 1], o[4 * jj + 2], o[4 * jj + 3]);
+              }
+            }
+            if (q_index >= 0) *reinterpret_cast<float2 *>(partial_ml + prow * 2) = make_float2(m_out, l_out);
+          }
+}
+
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map,
                const __grid_constant__ CUtensorMap q_map, DevBatch d, DevTcPlan tc, uint16_t *__restrict__ out,
@@ -431,6 +503,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant_
       mbar_init(&ctrl->drain[s], 1);
     }
     mbar_init(&ctrl->epi_done, 256);
+    mbar_init(&ctrl->xch, 128);
     ctrl->abort_flag = 0;
     fence_barrier_init();
   }
@@ -687,6 +760,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant_
     const uint32_t lane_base = tmem + ((uint32_t)(quarter * 32) << 16);
     const uint32_t s_addr = lane_base + s * 128, o_addr = lane_base + 256 + s * 128;
     uint32_t s_cnt = 0, o_cnt = 0;  // tiles / half-units of this stream so far
+    uint32_t x_cnt = 0;             // pieces so far in which the two streams were combined
     bool ok = true;
     for (int pc = piece0; pc < piece1; ++pc) {
       const TcPiece pi = pc == piece0 ? head->first : tc.pieces[pc];
@@ -803,43 +877,35 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant_
           o_cnt += 2u * (uint32_t)my_units;
           ok = wait_bar(&ctrl->o_done[s], (o_cnt - 1) & 1u, ctrl, d.status, 240 + s);
         }
-        if (ok) {
-          tc_fence_after();
-          const int slot = pi.slot[s];
-          if (slot < 0) {
-            const float inv = 1.0f / l;
-#pragma unroll
-            for (int hf = 0; hf < 2; ++hf) {
-              uint32_t o[64];
-              tmem_ld64(o_addr + hf * 64, o);
-              tc_wait_ld();
-              if (ri.q_index >= 0) {
-                uint4 *dst = reinterpret_cast<uint4 *>(out + ri.q_index * kD + hf * 64);
-#pragma unroll
-                for (int jj = 0; jj < 8; ++jj)
-                  dst[jj] = make_uint4(pack_bf16(bits_f(o[8 * jj]) * inv, bits_f(o[8 * jj + 1]) * inv),
-                                       pack_bf16(bits_f(o[8 * jj + 2]) * inv, bits_f(o[8 * jj + 3]) * inv),
-                                       pack_bf16(bits_f(o[8 * jj + 4]) * inv, bits_f(o[8 * jj + 5]) * inv),
-                                       pack_bf16(bits_f(o[8 * jj + 6]) * inv, bits_f(o[8 * jj + 7]) * inv));
-              }
-            }
-            if (lse != nullptr && ri.q_index >= 0) lse[ri.q_index] = (m_used + log2f(l)) * 0.6931471805599453f;
+        // The two streams of a one-M-tile piece hold partial results of the same rows (even and odd tiles).
+        // Stream 1 publishes its (m, l); stream 0 reads them and stream 1's accumulator -- the same tensor-memory
+        // lanes, so the thread of row r can load both -- and writes one combined result.
+        const bool pair = mode == 1 && n >= 2;
+        float m_out = m_used, l_out = l, w_self = 1.0f, w_other = 0.0f;
+        bool writer = true;
+        if (ok && pair) {
+          if (s == 1) {
+            ctrl->ml_xch[r] = make_float2(m_used, l);
+            tc_fence_before();
+            mbar_arrive(&ctrl->xch);
+            writer = false;
           } else {
-            const int64_t prow = (int64_t)slot * 128 + r;
-#pragma unroll
-            for (int hf = 0; hf < 2; ++hf) {
-              uint32_t o[64];
-              tmem_ld64(o_addr + hf * 64, o);
-              tc_wait_ld();
-              if (ri.q_index >= 0) {
-                // chunk-major: 16-byte chunk k of row r at [slot][k][r], so a warp's store is 512 contiguous bytes
-                uint4 *dst = reinterpret_cast<uint4 *>(tc.partial_o) + ((int64_t)slot * 32 + hf * 16) * 128 + r;
-#pragma unroll
-                for (int jj = 0; jj < 16; ++jj) dst[jj * 128] = make_uint4(o[4 * jj], o[4 * jj + 1], o[4 * jj + 2], o[4 * jj + 3]);
-              }
+            ok = wait_bar(&ctrl->xch, x_cnt & 1u, ctrl, d.status, 242);
+            if (ok) {
+              tc_fence_after();
+              const float2 other = ctrl->ml_xch[r];
+              m_out = fmaxf(m_used, other.x);
+              w_self = l > 0.f ? ex2(m_used - m_out) : 0.f;       // a stream that saw no key of the row has l = 0
+              w_other = other.y > 0.f ? ex2(other.x - m_out) : 0.f;
+              l_out = w_self * l + w_other * other.y;
             }
-            if (ri.q_index >= 0) *reinterpret_cast<float2 *>(tc.partial_ml + prow * 2) = make_float2(m_used, l);
           }
+        }
+        if (pair) ++x_cnt;
+        if (ok && writer) {
+          tc_fence_after();
+          store_rows(o_addr, lane_base + 256 + (1 - s) * 128, pi.slot[pair ? 0 : s], pair, w_self, w_other, m_out, l_out, r, ri.q_index, out,
+                     lse, tc.partial_o, tc.partial_ml);
           tc_fence_before();
         }
       }
@@ -993,6 +1059,25 @@ int tc_build_host_plan(const lr_ctx *ctx, const lr_batch *b, const int32_t *req_
   std::vector<TcReq> reqs((size_t)b->n_req);
   struct Grp { int req, kv, mtile0, n_mt, n_tiles, weight, first_piece, n_pieces; };
   std::vector<Grp> grps;
+  // Two M-tiles per group read every KV tile once for both, which is what a large pass needs.  A small pass --
+  // a few tiles per SM -- is dominated by the partial results of its key split instead; there every M-tile is a
+  // group of its own: a CTA then spends its two streams on the even and odd tiles of one M-tile, combines them
+  // on chip and writes one partial where the paired form writes two (the second reader of a KV tile finds it
+  // in L2).  Measured crossover: about 6 paired tiles per SM.
+  int m_step = 2;
+  {
+    int64_t paired = 0;
+    for (int r = 0; r < b->n_req; ++r) {
+      const int br0 = req_br_off[r], br1 = req_br_off[r + 1];
+      if (br1 == br0) continue;
+      int64_t n_pg = 0;
+      for (int sp = b->req_span_off[r]; sp < b->req_span_off[r + 1]; ++sp) n_pg += (b->span_len[sp] + kPage - 1) / kPage;
+      for (int i = br0; i < br1; ++i) n_pg += (b->br_own_len[i] + kPage - 1) / kPage;
+      const int64_t n_mt = (b->cu_q[br1] - b->cu_q[br0] + T - 1) / T;
+      paired += (n_pg + kPagesPerTile - 1) / kPagesPerTile * m.n_kv_heads * ((n_mt + 1) / 2);
+    }
+    if (paired <= 6 * (int64_t)ctx->sm_count) m_step = 1;
+  }
   for (int r = 0; r < b->n_req; ++r) {
     const int s0 = b->req_span_off[r], s1 = b->req_span_off[r + 1];
     const int br0 = req_br_off[r], br1 = req_br_off[r + 1];
@@ -1038,8 +1123,8 @@ int tc_build_host_plan(const lr_ctx *ctx, const lr_batch *b, const int32_t *req_
     const int n_tiles = (rq.n_pages + kPagesPerTile - 1) / kPagesPerTile;
     const int n_mtiles = (rq.n_q + T - 1) / T;
     for (int kv = 0; kv < m.n_kv_heads; ++kv)
-      for (int m0 = 0; m0 < n_mtiles; m0 += 2) {
-        const int mts = std::min(2, n_mtiles - m0);
+      for (int m0 = 0; m0 < n_mtiles; m0 += m_step) {
+        const int mts = std::min(m_step, n_mtiles - m0);
         grps.push_back(Grp{r, kv, m0, mts, n_tiles, 1 + mts, 0, 0});
       }
   }
@@ -1119,12 +1204,8 @@ int tc_build_host_plan(const lr_ctx *ctx, const lr_batch *b, const int32_t *req_
       std::vector<int32_t *> contrib;
       for (int k = 0; k < g.n_pieces; ++k) {
         TcPiece &p = pieces[g.first_piece + k];
-        const int n = p.tile_end - p.tile_begin;
         if (g.n_mt == 2) contrib.push_back(&p.slot[mt]);
-        else {
-          contrib.push_back(&p.slot[0]);
-          if (n >= 2) contrib.push_back(&p.slot[1]);
-        }
+        else contrib.push_back(&p.slot[0]);  // the two streams of a one-M-tile piece are combined inside the CTA
       }
       if (contrib.size() == 1) { *contrib[0] = -1; continue; }
       TcTarget tg;
