@@ -101,6 +101,7 @@ accept_greedy_kernel(const uint16_t *__restrict__ logits, int64_t row_stride, in
   __shared__ int32_t s_i[kThreads / 32];
   __shared__ int s_last;
   asm volatile("griddepcontrol.wait;" ::: "memory");  // the logits may come from the kernel launched just before
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");  // lr_commit's grid may be set up meanwhile
 
   while (pos < end) {
     const int row = (int)(pos / upr);

@@ -65,6 +65,7 @@ commit_kernel(DevBatch d, const uint8_t *__restrict__ verdict,
   __shared__ int32_t s_total[2];
   const int tid = threadIdx.x;
   asm volatile("griddepcontrol.wait;" ::: "memory");  // n_accept comes from the kernel launched just before
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
   // ---- per-request decisions --------------------------------------------------
   for (int r = tid; r < R; r += kThreads) {
@@ -186,6 +187,7 @@ commit_tree_kernel(DevBatch d, const uint8_t *__restrict__ verdict,
   __shared__ int32_t s_total[2];
   const int tid = threadIdx.x;
   asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
   for (int r = tid; r < R; r += kThreads) {
     const int s0 = d.req_span_off[r], s1 = d.req_span_off[r + 1];
@@ -314,14 +316,14 @@ int launch_commit(lr_plan *p, const uint8_t *verdict, const int32_t *n_accept, i
   grid = grid < 1 ? 1 : (grid > cap ? cap : grid);
   p->ctx->launches++;
   if (d.tree) {
-    commit_tree_kernel<<<grid, kThreads, (size_t)d.n_req * kSmemPerReqTree, s>>>(
-        d, verdict, n_accept, n_steps, survivor, committed, keep_off, keep_pages, keep_valid, free_off, free_pages);
-    return cuda_fail(cudaGetLastError(), "commit_tree_kernel launch");
+    return cuda_fail(launch_dependent(commit_tree_kernel, dim3(grid), dim3(kThreads), (size_t)d.n_req * kSmemPerReqTree, s, d, verdict,
+                                      n_accept, n_steps, survivor, committed, keep_off, keep_pages, keep_valid, free_off, free_pages),
+                     "commit_tree_kernel launch");
   }
   size_t smem = (size_t)d.n_req * kSmemPerReq;
-  commit_kernel<<<grid, kThreads, smem, s>>>(d, verdict, n_accept, n_steps, survivor, committed,
-                                              keep_off, keep_pages, keep_valid, free_off, free_pages);
-  return cuda_fail(cudaGetLastError(), "commit_kernel launch");
+  return cuda_fail(launch_dependent(commit_kernel, dim3(grid), dim3(kThreads), smem, s, d, verdict, n_accept, n_steps, survivor, committed,
+                                    keep_off, keep_pages, keep_valid, free_off, free_pages),
+                   "commit_kernel launch");
 }
 
 }  // namespace lr
