@@ -7,10 +7,12 @@
 // stay where they are.  Three small kernels:
 //   compact_scan_kernel     one CTA per request: exclusive scan of the valid counts of its kept pages
 //                           (token offset of every page), the new length, the first displaced page;
-//   compact_move_kernel<0>  one CTA per kept page: its tokens -> staging[token index]   (gather);
-//   compact_move_kernel<1>  one CTA per kept page: staging -> destination page and slot (scatter).
+//   compact_move_kernel<0>  a fixed grid over the displaced pages: tokens -> staging[token index]      (gather);
+//   compact_move_kernel<1>  the same walk: staging -> destination page and slot                      (scatter).
 // Bytes moved: 2 (K, V) x H_kv x D x 2 B per displaced token, read and written twice; the work is bound by
 // the latency of three dependent launches, not by bandwidth.
+#include <algorithm>
+
 #include "lr_common.cuh"
 
 namespace lr {
@@ -18,6 +20,7 @@ namespace lr {
 namespace {
 
 constexpr int kThreads = 256;
+constexpr int kMaxReq = 8192;  // the move kernels keep one prefix sum per request in shared memory
 
 __global__ void __launch_bounds__(kThreads)
 compact_scan_kernel(const int32_t *__restrict__ keep_off, const int32_t *__restrict__ keep_valid, int32_t *__restrict__ tok_off,
@@ -62,63 +65,93 @@ compact_scan_kernel(const int32_t *__restrict__ keep_off, const int32_t *__restr
   }
 }
 
-// request of kept-list entry i: largest r with keep_off[r] <= i
-__device__ __forceinline__ int find_request(const int32_t *keep_off, int n_req, int i) {
-  int lo = 0, hi = n_req - 1;
-  while (lo < hi) {
-    const int mid = (lo + hi + 1) >> 1;
-    if (keep_off[mid] <= i) lo = mid; else hi = mid - 1;
-  }
-  return lo;
-}
-
-// kScatter = false: pools -> staging; true: staging -> pools.  One CTA per entry of the keep lists.
+// kScatter = false: pools -> staging; true: staging -> pools.  A fixed grid walks the displaced entries of the keep
+// lists only: request r has keep_off[r+1] - first_moved[r] of them (none when nothing of it moves); every CTA builds
+// the prefix sums of those counts in shared memory and takes the work items blockIdx.x, blockIdx.x + gridDim.x, ...
 template <bool kScatter>
 __global__ void __launch_bounds__(kThreads)
 compact_move_kernel(DevBatch d, const int32_t *__restrict__ keep_off, const int32_t *__restrict__ keep_pages,
                     const int32_t *__restrict__ keep_valid, const int32_t *__restrict__ tok_off,
                     const int32_t *__restrict__ first_moved, const int32_t *__restrict__ stage_off, uint4 *__restrict__ k_pool,
                     uint4 *__restrict__ v_pool, uint4 *__restrict__ staging) {
-  const int i = blockIdx.x;
+  extern __shared__ int32_t s_off[];  // [n_req + 1] displaced entries in front of request r
+  __shared__ int32_t warp_sum[kThreads / 32];
+  __shared__ int32_t s_carry;
+  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
   asm volatile("griddepcontrol.wait;" ::: "memory");
-  if (i >= keep_off[d.n_req]) return;
-  const int r = find_request(keep_off, d.n_req, i);
-  const int f = first_moved[r];
-  if (i < f) return;  // not displaced
-  const int valid = keep_valid[i];
-  const int64_t src_page = keep_pages[i];
-  const int k0_chk = tok_off[i] - tok_off[f];
-  if (src_page < 0 || src_page >= d.n_pool_pages || valid < 0 || valid > kPage ||
-      k0_chk + valid > stage_off[r + 1] - stage_off[r]) {  // never touch memory outside the pools or the staging area
-    if (threadIdx.x == 0) {
-      d.status[0] = kDevBounds;
-      d.status[1] = 400;
+  if (tid == 0) s_carry = 0;
+  __syncthreads();
+  for (int base = 0; base < d.n_req; base += kThreads) {
+    const int r = base + tid;
+    const int32_t x = r < d.n_req ? min(d.n_page_slots, max(0, keep_off[r + 1] - first_moved[r])) : 0;
+    int32_t inc = x;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int32_t y = __shfl_up_sync(0xFFFFFFFFu, inc, o);
+      if (lane >= o) inc += y;
     }
-    return;
+    if (lane == 31) warp_sum[wid] = inc;
+    __syncthreads();
+    int32_t wbase = 0;
+    for (int w = 0; w < wid; ++w) wbase += warp_sum[w];
+    const int32_t carry = s_carry;
+    if (r < d.n_req) s_off[r] = carry + wbase + inc - x;
+    __syncthreads();
+    if (tid == kThreads - 1) s_carry = carry + wbase + inc;
+    __syncthreads();
   }
-  const int i0 = keep_off[r];
-  const int k0 = tok_off[i];                      // committed-sequence index of the page's first token
-  const int m0 = k0 - tok_off[f];                 // index among the request's displaced tokens
-  const int vec_per_row = d.head_dim / 8;         // 16-byte vectors per (token, head)
-  const int per_tok = d.n_kv_heads * vec_per_row; // per pool
-  for (int idx = threadIdx.x; idx < valid * per_tok; idx += kThreads) {
-    const int t = idx / per_tok, rem = idx - t * per_tok, h = rem / vec_per_row, c = rem - h * vec_per_row;
-    const int64_t s_idx = ((int64_t)(stage_off[r] + m0 + t) * 2) * per_tok + rem;  // [token][K, V][head][vector]
-    if (!kScatter) {
-      const int64_t src = ((src_page * d.n_kv_heads + h) * kPage + t) * vec_per_row + c;
-      staging[s_idx] = k_pool[src];
-      staging[s_idx + per_tok] = v_pool[src];
-    } else {
-      const int k = k0 + t;
-      const int64_t dst_page = keep_pages[i0 + k / kPage];
-      if (dst_page < 0 || dst_page >= d.n_pool_pages) {
+  const int32_t total = s_carry;
+  if (tid == 0) s_off[d.n_req] = total;
+  __syncthreads();
+  const int vec_per_row = d.head_dim / 8;          // 16-byte vectors per (token, head)
+  const int per_tok = d.n_kv_heads * vec_per_row;  // per pool
+  for (int32_t w = blockIdx.x; w < total; w += gridDim.x) {
+    int lo = 0, hi = d.n_req - 1;  // request of work item w: largest r with s_off[r] <= w (requests without items are skipped)
+    while (lo < hi) {
+      const int mid = (lo + hi + 1) >> 1;
+      if (s_off[mid] <= w) lo = mid; else hi = mid - 1;
+    }
+    const int r = lo;
+    const int f = first_moved[r], i = f + (w - s_off[r]);
+    if (f < 0 || i < 0 || i >= d.n_page_slots) {  // keep lists that do not come from lr_commit
+      if (tid == 0) {
         d.status[0] = kDevBounds;
-        d.status[1] = 401;
-        continue;
+        d.status[1] = 402;
       }
-      const int64_t dst = ((dst_page * d.n_kv_heads + h) * kPage + (k % kPage)) * vec_per_row + c;
-      k_pool[dst] = staging[s_idx];
-      v_pool[dst] = staging[s_idx + per_tok];
+      continue;
+    }
+    const int valid = keep_valid[i];
+    const int64_t src_page = keep_pages[i];
+    const int m0 = tok_off[i] - tok_off[f];  // index among the request's displaced tokens
+    if (src_page < 0 || src_page >= d.n_pool_pages || valid < 0 || valid > kPage ||
+        m0 + valid > stage_off[r + 1] - stage_off[r]) {  // never touch memory outside the pools or the staging area
+      if (tid == 0) {
+        d.status[0] = kDevBounds;
+        d.status[1] = 400;
+      }
+      continue;
+    }
+    const int i0 = keep_off[r];
+    const int k0 = tok_off[i];  // committed-sequence index of the page's first token
+    for (int idx = tid; idx < valid * per_tok; idx += kThreads) {
+      const int t = idx / per_tok, rem = idx - t * per_tok, h = rem / vec_per_row, c = rem - h * vec_per_row;
+      const int64_t s_idx = ((int64_t)(stage_off[r] + m0 + t) * 2) * per_tok + rem;  // [token][K, V][head][vector]
+      if (!kScatter) {
+        const int64_t src = ((src_page * d.n_kv_heads + h) * kPage + t) * vec_per_row + c;
+        staging[s_idx] = k_pool[src];
+        staging[s_idx + per_tok] = v_pool[src];
+      } else {
+        const int k = k0 + t;
+        const int64_t dst_page = keep_pages[i0 + k / kPage];
+        if (dst_page < 0 || dst_page >= d.n_pool_pages) {
+          d.status[0] = kDevBounds;
+          d.status[1] = 401;
+          continue;
+        }
+        const int64_t dst = ((dst_page * d.n_kv_heads + h) * kPage + (k % kPage)) * vec_per_row + c;
+        k_pool[dst] = staging[s_idx];
+        v_pool[dst] = staging[s_idx + per_tok];
+      }
     }
   }
 }
@@ -136,12 +169,17 @@ int launch_compact(lr_plan *p, const int32_t *keep_off, const int32_t *keep_page
   compact_scan_kernel<<<d.n_req, kThreads, 0, s>>>(keep_off, keep_valid, tok_off, first_moved, new_len, n_pages_kept);
   p->ctx->launches++;
   if (int rc = cuda_fail(cudaGetLastError(), "compact_scan_kernel launch")) return rc;
-  const unsigned grid = (unsigned)d.n_page_slots;  // upper bound of the keep lists
-  compact_move_kernel<false><<<grid, kThreads, 0, s>>>(d, keep_off, keep_pages, keep_valid, tok_off, first_moved, stage_off,
+  if (d.n_req > kMaxReq) {
+    set_error("lr_compact: more than %d requests in one pass", kMaxReq);
+    return LR_EUNSUPPORTED;
+  }
+  const unsigned grid = (unsigned)std::max(1, std::min(d.n_page_slots, p->ctx->sm_count * 8));
+  const size_t smem = sizeof(int32_t) * ((size_t)d.n_req + 1);
+  compact_move_kernel<false><<<grid, kThreads, smem, s>>>(d, keep_off, keep_pages, keep_valid, tok_off, first_moved, stage_off,
                                                       reinterpret_cast<uint4 *>(k_pool), reinterpret_cast<uint4 *>(v_pool), staging);
   p->ctx->launches++;
   if (int rc = cuda_fail(cudaGetLastError(), "compact gather launch")) return rc;
-  compact_move_kernel<true><<<grid, kThreads, 0, s>>>(d, keep_off, keep_pages, keep_valid, tok_off, first_moved, stage_off,
+  compact_move_kernel<true><<<grid, kThreads, smem, s>>>(d, keep_off, keep_pages, keep_valid, tok_off, first_moved, stage_off,
                                                      reinterpret_cast<uint4 *>(k_pool), reinterpret_cast<uint4 *>(v_pool), staging);
   p->ctx->launches++;
   return cuda_fail(cudaGetLastError(), "compact scatter launch");
