@@ -105,8 +105,11 @@ compact_move_kernel(DevBatch d, const int32_t *__restrict__ keep_off, const int3
   __syncthreads();
   const int vec_per_row = d.head_dim / 8;          // 16-byte vectors per (token, head)
   const int per_tok = d.n_kv_heads * vec_per_row;  // per pool
-  for (int32_t w = blockIdx.x; w < total; w += gridDim.x) {
-    int lo = 0, hi = d.n_req - 1;  // request of work item w: largest r with s_off[r] <= w (requests without items are skipped)
+  // a work item is one KV head of one displaced page (8 KB of K and V): enough items to spread a few hundred pages
+  for (int64_t item = blockIdx.x; item < (int64_t)total * d.n_kv_heads; item += gridDim.x) {
+    const int32_t w = (int32_t)(item / d.n_kv_heads);
+    const int h = (int)(item - (int64_t)w * d.n_kv_heads);
+    int lo = 0, hi = d.n_req - 1;  // request of page w: largest r with s_off[r] <= w (requests without items are skipped)
     while (lo < hi) {
       const int mid = (lo + hi + 1) >> 1;
       if (s_off[mid] <= w) lo = mid; else hi = mid - 1;
@@ -133,8 +136,8 @@ compact_move_kernel(DevBatch d, const int32_t *__restrict__ keep_off, const int3
     }
     const int i0 = keep_off[r];
     const int k0 = tok_off[i];  // committed-sequence index of the page's first token
-    for (int idx = tid; idx < valid * per_tok; idx += kThreads) {
-      const int t = idx / per_tok, rem = idx - t * per_tok, h = rem / vec_per_row, c = rem - h * vec_per_row;
+    for (int idx = tid; idx < valid * vec_per_row; idx += kThreads) {
+      const int t = idx / vec_per_row, c = idx - t * vec_per_row, rem = h * vec_per_row + c;
       const int64_t s_idx = ((int64_t)(stage_off[r] + m0 + t) * 2) * per_tok + rem;  // [token][K, V][head][vector]
       if (!kScatter) {
         const int64_t src = ((src_page * d.n_kv_heads + h) * kPage + t) * vec_per_row + c;
@@ -173,7 +176,7 @@ int launch_compact(lr_plan *p, const int32_t *keep_off, const int32_t *keep_page
     set_error("lr_compact: more than %d requests in one pass", kMaxReq);
     return LR_EUNSUPPORTED;
   }
-  const unsigned grid = (unsigned)std::max(1, std::min(d.n_page_slots, p->ctx->sm_count * 8));
+  const unsigned grid = (unsigned)std::max<int64_t>(1, std::min<int64_t>((int64_t)d.n_page_slots * d.n_kv_heads, p->ctx->sm_count * 4));
   const size_t smem = sizeof(int32_t) * ((size_t)d.n_req + 1);
   compact_move_kernel<false><<<grid, kThreads, smem, s>>>(d, keep_off, keep_pages, keep_valid, tok_off, first_moved, stage_off,
                                                       reinterpret_cast<uint4 *>(k_pool), reinterpret_cast<uint4 *>(v_pool), staging);
