@@ -672,8 +672,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant_
           if (my_units == 1) tc_commit(&ctrl->q_empty);  // last QK of the piece: this stream is done with the Q buffers
         }
         __syncwarp();
-      } else if (lane == 0) {
-        mbar_arrive(&ctrl->q_empty);
+      } else {
+        if (lane == 0) mbar_arrive(&ctrl->q_empty);
+        // nothing to issue in this piece: still observe the previous piece's epilogue phase, so that the parity
+        // wait of a later piece never finds this issuer two phases behind
+        if (pc_idx > 0) {
+          ok = wait_bar(&ctrl->epi_done, (pc_idx - 1) & 1u, ctrl, d.status, 228);
+          if (!ok) break;
+        }
       }
       for (int j = 0; j < my_units && ok; ++j) {
         const int t = mode == 2 ? j : 2 * j + s;
@@ -909,6 +915,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant_
           tc_fence_before();
         }
       }
+      // One arrival per thread and piece.  A stream with units in this piece cannot get here before the previous
+      // piece's phase is complete (its PV products were issued behind a wait for it); a stream with none must look
+      // itself, or its arrival would be counted into the previous phase while the other stream is still storing.
+      if (my_units == 0 && pc > piece0 && ok) ok = wait_bar(&ctrl->epi_done, (uint32_t)(pc - piece0 - 1) & 1u, ctrl, d.status, 243);
       mbar_arrive(&ctrl->epi_done);
     }
   }

@@ -28,6 +28,14 @@ def test_whole_pass_random_trees_tensor_core_path(seed):
     run_and_check_pass(make_random_tree(600 + seed, head_dim=128))
 
 
+def test_many_small_passes_on_the_tensor_core_path():
+    """Tiny passes put several one-tile pieces into one CTA, where one of its two streams has nothing to do: the
+    piece-by-piece barrier phases must still line up (seed 5000 once ran into an expired wait)."""
+    for seed in [5000] + list(range(5100, 5140)):
+        run_and_check_pass(make_random_tree(seed, head_dim=128))
+        run_and_check_pass(make_random_small(seed, head_dim=128))
+
+
 @pytest.mark.parametrize("seed", list(range(4)))
 def test_whole_pass_random_trees_generic_path(seed):
     run_and_check_pass(make_random_tree(700 + seed), path=B.PATH_GENERIC)
