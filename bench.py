@@ -449,7 +449,7 @@ def main():
         roof["frac"] = roof["achieved"] / roof["peak"]
         # dram__bytes_read.sum + dram__bytes_write.sum of one attn_tc_kernel launch on this workload (ncu
         # captures summarised under profiles/, taken on the kernels as they are); None where not captured
-        traffic = ({2: 17_980_672 + 0, 3: 275_110_144 + 6_377_472}.get(args.config)
+        traffic = ({2: 17_981_696 + 0, 3: 275_153_152 + 7_003_648}.get(args.config)
                    if args.path == 0 and not args.carry_in and not args.tree else None)
         roof.update({"traffic": traffic, "kernel": "lr_verify_attention", "kernel_us": kernel_us["attention"],
                      "algorithmic_bytes": a_bytes, "algorithmic_flops": a_flops, "peak_source": f"of {peak_kind}", "timed": "attn_tc_kernel + attn_tc_merge_kernel",
