@@ -22,4 +22,5 @@ from .gen import (  # noqa: F401
     make_random_small,
     make_tree,
     make_random_tree,
+    make_random_mid,
 )

@@ -531,3 +531,28 @@ def make_random_tree(seed: int, head_dim: Optional[int] = None, poison: str = "n
             branches.append((int(rng.integers(0, n + 1)), own_len, q_len, n_draft))
         reqs.append({"P": P, "segs": segs, "parents": parents, "branches": branches})
     return _finish(f"random_tree_{seed}", seed, model, reqs, rng, 0.3, 0.6, True, True, poison)
+
+
+def make_random_mid(seed: int) -> Workload:
+    """Mid-size ragged batches (1-6 requests, contexts of 100-6000 tokens, 1-5 draft steps as a chain or a tree,
+    several head geometries with head_dim 128): a few to a few dozen key tiles per SM, i.e. both sides of the point
+    where the attention plan switches between its two ways of grouping query tiles."""
+    rng = np.random.Generator(np.random.PCG64(9000 + seed))
+    hq, hkv = [(40, 8), (16, 4), (8, 8), (32, 8), (5, 1)][seed % 5]
+    model = Model(hq, hkv, 128, int(rng.choice([1000, 4099])))
+    reqs = []
+    for _ in range(int(rng.integers(1, 7))):
+        gamma = int(rng.integers(1, 6))
+        L = int(rng.choice([4, 8, 16]))
+        req = {"P": int(rng.integers(100, 6000)), "segs": [int(v) for v in rng.integers(8, 80, size=gamma)]}
+        if rng.random() < 0.4:
+            req["parents"] = [int(rng.integers(0, c + 1)) for c in range(gamma)]
+            req["branches"] = ([(n, L + int(rng.choice([0, 3])), L, L) for n in range(gamma + 1) if rng.random() < 0.8]
+                               or [(0, L, L, L)])
+        else:
+            req["branches"] = [(j, L, L, L) for j in range(1, gamma + 1)]
+        reqs.append(req)
+    if any("parents" in r for r in reqs):  # one batch is a chain batch or a tree batch
+        for r in reqs:
+            r.setdefault("parents", list(range(len(r["segs"]))))
+    return _finish(f"random_mid_{seed}", seed, model, reqs, rng, 0.3, 0.6, True, True, "nan")

@@ -5,7 +5,7 @@ import numpy as np
 import pytest
 import torch
 
-from lr_workloads import Model, bf16_round, build_batch, fill_kv, fill_q, make_config, make_random_small
+from lr_workloads import Model, bf16_round, build_batch, fill_kv, fill_q, make_config, make_random_mid, make_random_small
 from oracle import lr_oracle as O
 from paper_2506_19830_b200 import binding as B
 from paper_2506_19830_b200 import runner as R
@@ -47,6 +47,16 @@ def test_whole_pass_with_the_carry_in_token_as_a_query(cfg):
 @pytest.mark.parametrize("seed", list(range(16)))
 def test_whole_pass_ragged_small(seed):
     run_and_check_pass(make_random_small(1000 + seed))
+
+
+@pytest.mark.parametrize("seed", list(range(10)))
+def test_whole_pass_mid_size_batches(seed):
+    """Both sides of the attention plan's switch between pairing query tiles and taking them one by one; attention is
+    compared on a sample of branches (the oracle is slow), acceptance and commit in full."""
+    w = make_random_mid(seed)
+    rng = _rng(seed)
+    pick = sorted(set(int(x) for x in rng.integers(0, w.batch.n_branch, size=min(4, w.batch.n_branch))))
+    run_and_check_pass(w, check_rows_of_branches=pick)
 
 
 def test_overlapped_pass_gives_the_same_results():
