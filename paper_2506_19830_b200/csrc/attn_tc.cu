@@ -34,7 +34,7 @@
 //               the MMA descriptors read with SBO = 2048.  One box per page rather
 //               than one per page half matters: the producer spends about 100
 //               cycles per box, and 32 boxes per tile made it a bottleneck.
-//               No multicast.
+//               Every copy is for this CTA alone.
 //   warps 9, 10 MMA issuers of stream 0 and 1 (warp 11 idles): tcgen05.mma (M=128, N=128, K=16,
 //               bf16 -> fp32) for S = Q K^T (both operands in shared memory) and
 //               O += P V (P read from tensor memory, V from shared memory as the
@@ -159,7 +159,7 @@ __device__ __forceinline__ void tc_commit(uint64_t *bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 
-// Tiled bulk tensor copies global -> shared, completion on an mbarrier (no multicast).
+// Tiled bulk tensor copies global -> shared for this CTA alone, completion on an mbarrier.
 __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *map, int32_t x, int32_t y, int32_t z, int32_t w, uint64_t *bar) {
   asm volatile(
       "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];" ::"r"(dst),
