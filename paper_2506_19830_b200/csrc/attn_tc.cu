@@ -1053,7 +1053,7 @@ int init_attn_tc_kernel() {
 
 // ---- host planning -----------------------------------------------------------------
 // most CTAs worth using for a number of tiles (tiny problems: not one CTA per tile, their partial results cost more than they save)
-static int64_t kCtaPerTiles(int64_t tiles) { return tiles >= 64 ? tiles : tiles / 2; }
+static int64_t max_ctas_for_tiles(int64_t tiles) { return tiles >= 64 ? tiles : tiles / 2; }
 
 int tc_build_host_plan(const lr_ctx *ctx, const lr_batch *b, const int32_t *req_br_off, const int32_t *span_tin,
                        const int32_t *span_last, TcHostPlan &out, Image &img) {
@@ -1156,7 +1156,7 @@ int tc_build_host_plan(const lr_ctx *ctx, const lr_batch *b, const int32_t *req_
     total_tiles += g.n_tiles;
     lo = std::max<int64_t>(lo, (int64_t)(kPieceStartTiles * kDense + kMasked) * g.weight);
   }
-  const int64_t max_cta = std::min<int64_t>(ctx->sm_count, std::max<int64_t>(1, kCtaPerTiles(total_tiles)));
+  const int64_t max_cta = std::min<int64_t>(ctx->sm_count, std::max<int64_t>(1, max_ctas_for_tiles(total_tiles)));
   // walks the partition for limit L; with `emit` it also records the pieces.  A group is a run of dense tiles
   // followed by a run of masked ones, each of uniform cost, so a walk takes O(CTAs + groups) steps.
   std::vector<TcPiece> pieces;
