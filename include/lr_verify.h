@@ -163,11 +163,33 @@ int lr_plan_destroy(lr_plan *plan);
 int lr_verify_attention(lr_plan *plan, const void *q_d, const void *k_pool_d, const void *v_pool_d,
                         void *out_d, float *lse_d, float softmax_scale, void *stream);
 
+/* What lr_verify_attention will launch for this plan (host-side query, no device work).
+ *   tensor_core_ok   1 when the shape allows the tcgen05 kernel (head_dim 128, tensor-map coordinates
+ *                    within 32 bits, at most 254 branches per request, tails of at most 2047 pages)
+ *   path             the current selection (0 automatic, 1 CUDA cores, 2 tensor cores)
+ *   uses_tensor_core 1 when the next call would run the tcgen05 kernel
+ *   n_cta            CTAs of the tcgen05 kernel (0 on the CUDA-core path)
+ *   n_pieces         (CTA, request, KV head, query tiles) work items
+ *   n_merge_targets  query tiles whose keys are split over several CTAs and need a merge
+ *   n_partial_slots  fp32 partial results those CTAs write
+ */
+typedef struct lr_plan_info {
+  int32_t tensor_core_ok, path, uses_tensor_core, n_cta, n_pieces, n_merge_targets, n_partial_slots;
+} lr_plan_info;
+int lr_plan_describe(const lr_plan *plan, lr_plan_info *info_out);
+
 /* Selects the attention implementation for later lr_verify_attention calls on
  * this plan: 0 = automatic (tensor-core path when the shape allows it), 1 =
  * force the CUDA-core path (every shape), 2 = force the tensor-core path
  * (LR_EUNSUPPORTED later if the shape does not allow it).  For testing. */
 int lr_plan_set_attention_path(lr_plan *plan, int path);
+
+/* Test hook for the device-side bounds checks: overwrites the physical page id of page slot `page_slot`
+ * (an index into lr_batch.page_ids) with new_id in every device table of the plan, by patching the plan's host
+ * image and uploading it again on `stream`.  No validation of new_id: that is the point.  A kernel that meets
+ * an id outside [0, n_pool_pages) reads page 0 in its place and raises LR_EBOUNDS in the status word
+ * (lr_poll_status); it never dereferences the id. */
+int lr_plan_debug_set_page(lr_plan *plan, int32_t page_slot, int32_t new_id, void *stream);
 
 /* Bytes of scratch lr_accept_greedy needs for n_rows logits rows.  The scratch
  * must be zero-filled before its first use; every call leaves it zero-filled. */
@@ -233,7 +255,10 @@ int lr_accept_sample(lr_ctx *ctx, const void *logits_d, int64_t row_stride_elems
  *   - n_rows > LR_ACCEPT_STATIC_MAX_ROWS is rejected with LR_EINVAL.
  *   - The first call on a device looks up the array's device address (a
  *     cudaGetSymbolAddress call, made with ctx's device current); make that
- *     first call outside any stream capture.
+ *     first call outside any stream capture, and from one thread only (the
+ *     looked-up address is cached without a lock).
+ *   - Every call makes ctx's device current for its own duration and puts the
+ *     caller's current device back before it returns.
  *   - All calls on one device share the one array.  Each call clears the part
  *     it uses on `stream` before its kernel runs, so leftovers of an earlier
  *     call never matter, but two calls whose device work overlaps in time
@@ -269,7 +294,12 @@ int lr_accept_greedy_static(lr_ctx *ctx, const void *logits_d, int64_t row_strid
  * lowest-numbered branch that continues the node reached, the kept segments
  * are those moved through (keep list in that order) and the free list holds
  * every other segment in index order, then the tails as above.
+ *
+ * At most LR_COMMIT_MAX_REQUESTS requests per pass: a plan of a larger batch is
+ * accepted (attention and acceptance have no such limit) but lr_commit on it
+ * returns LR_EUNSUPPORTED before anything is launched.
  */
+#define LR_COMMIT_MAX_REQUESTS 4096
 int lr_commit(lr_plan *plan, const uint8_t *verdict_d, const int32_t *n_accept_d,
               int32_t *n_steps_accepted_d, int32_t *survivor_d, int32_t *committed_len_d,
               int32_t *keep_off_d, int32_t *keep_pages_d, int32_t *keep_valid_d,
@@ -289,8 +319,11 @@ int lr_commit(lr_plan *plan, const uint8_t *verdict_d, const int32_t *n_accept_d
  * scratch_d: lr_compact_scratch_bytes bytes, 256-byte aligned, no initial
  * contents needed.  Three launches on `stream`; a page id outside the pools sets
  * the plan's status word (LR_EBOUNDS) instead of being dereferenced.  The batch
- * must be the one the plan and the keep lists were made for.
+ * must be the one the plan and the keep lists were made for.  At most
+ * LR_COMPACT_MAX_REQUESTS requests per pass (LR_EUNSUPPORTED beyond, before
+ * anything is launched or written).
  */
+#define LR_COMPACT_MAX_REQUESTS 8192
 int lr_compact_scratch_bytes(const lr_plan *plan, size_t *bytes_out);
 int lr_compact(lr_plan *plan, const int32_t *keep_off_d, const int32_t *keep_pages_d, const int32_t *keep_valid_d,
                void *k_pool_d, void *v_pool_d, int32_t *new_len_d, int32_t *n_pages_kept_d, void *scratch_d, void *stream);

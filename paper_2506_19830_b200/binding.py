@@ -23,6 +23,8 @@ STATUS_NAMES = {0: "LR_OK", -1: "LR_EINVAL", -2: "LR_EUNSUPPORTED", -3: "LR_ECUD
 
 PATH_AUTO, PATH_GENERIC, PATH_TENSOR_CORE = 0, 1, 2
 ACCEPT_STATIC_MAX_ROWS = 4096  # LR_ACCEPT_STATIC_MAX_ROWS
+COMMIT_MAX_REQUESTS = 4096  # LR_COMMIT_MAX_REQUESTS
+COMPACT_MAX_REQUESTS = 8192  # LR_COMPACT_MAX_REQUESTS
 
 
 class LrError(RuntimeError):
@@ -48,6 +50,11 @@ class lr_batch(C.Structure):
 
 class lr_cycle_stats(C.Structure):
     _fields_ = [(n, C.c_int64) for n in ("stages", "steps", "time", "verdicts_used", "peak_in_flight")]
+
+
+class lr_plan_info(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("tensor_core_ok", "path", "uses_tensor_core", "n_cta", "n_pieces",
+                                         "n_merge_targets", "n_partial_slots")]
 
 
 class lr_pass_host_io(C.Structure):
@@ -77,6 +84,8 @@ def lib() -> C.CDLL:
             "lr_plan_create": [vp, C.POINTER(lr_batch), vp, sz, vp, C.POINTER(vp)],
             "lr_plan_destroy": [vp],
             "lr_plan_set_attention_path": [vp, C.c_int],
+            "lr_plan_describe": [vp, C.POINTER(lr_plan_info)],
+            "lr_plan_debug_set_page": [vp, i32, i32, vp],
             "lr_verify_attention": [vp, vp, vp, vp, vp, vp, f32, vp],
             "lr_accept_scratch_bytes": [i32, C.POINTER(sz)],
             "lr_accept_greedy": [vp, vp, i64, vp, vp, i32, i32, vp, vp, vp, vp, vp],
@@ -265,6 +274,14 @@ class Plan:
 
     def lr_plan_set_attention_path(self, path: int) -> None:
         _check(lib().lr_plan_set_attention_path(self.handle, path), "lr_plan_set_attention_path")
+
+    def lr_plan_debug_set_page(self, page_slot: int, new_id: int, stream=None) -> None:
+        _check(lib().lr_plan_debug_set_page(self.handle, page_slot, new_id, _stream_ptr(stream)), "lr_plan_debug_set_page")
+
+    def lr_plan_describe(self) -> dict:
+        info = lr_plan_info()
+        _check(lib().lr_plan_describe(self.handle, C.byref(info)), "lr_plan_describe")
+        return {n: int(getattr(info, n)) for n, _ in lr_plan_info._fields_}
 
     def lr_verify_attention(self, q, k_pool, v_pool, out, lse=None, softmax_scale: float = 0.0, stream=None) -> None:
         _check(lib().lr_verify_attention(self.handle, _ptr(q), _ptr(k_pool), _ptr(v_pool), _ptr(out), _ptr(lse),

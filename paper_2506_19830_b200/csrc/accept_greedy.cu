@@ -247,17 +247,28 @@ int launch_accept_static(lr_ctx *ctx, const void *logits, int64_t stride, const 
     set_error("lr_accept_greedy_static: device ordinal %d not supported", ctx->device);
     return LR_EUNSUPPORTED;
   }
-  if (int rc = cuda_fail(cudaSetDevice(ctx->device), "cudaSetDevice")) return rc;
+  // ctx's device is made current for the symbol look-up and the launch; the caller's own choice is put back afterwards
+  int prev_device = -1;
+  if (int rc = cuda_fail(cudaGetDevice(&prev_device), "cudaGetDevice")) return rc;
+  if (prev_device != ctx->device)
+    if (int rc = cuda_fail(cudaSetDevice(ctx->device), "cudaSetDevice")) return rc;
+  int rc = LR_OK;
   void *ptr = g_static_scratch_addr[ctx->device];
   if (ptr == nullptr) {
     // In host code the array's name is only a handle; the kernel needs the address the symbol has
-    // on *this* device.  Done once per device, with that device current.
-    if (int rc = cuda_fail(cudaGetSymbolAddress(&ptr, g_static_scratch), "cudaGetSymbolAddress(static scratch)")) return rc;
-    g_static_scratch_addr[ctx->device] = ptr;
+    // on *this* device.  Done once per device, with that device current.  The cache is written without a
+    // lock (every writer stores the same value); the first call per device should still come from one thread.
+    rc = cuda_fail(cudaGetSymbolAddress(&ptr, g_static_scratch), "cudaGetSymbolAddress(static scratch)");
+    if (rc == LR_OK) g_static_scratch_addr[ctx->device] = ptr;
   }
   // Every call shares the array and it keeps what the last call left: start from zero regardless.
-  if (int rc = cuda_fail(cudaMemsetAsync(ptr, 0, 8 * ((size_t)n_rows + 1), s), "cudaMemsetAsync(static scratch)")) return rc;
-  return launch_accept(ctx, logits, stride, drafts, cu_draft, n_branch, n_rows, n_accept, bonus, row_argmax, ptr, s);
+  if (rc == LR_OK) rc = cuda_fail(cudaMemsetAsync(ptr, 0, 8 * ((size_t)n_rows + 1), s), "cudaMemsetAsync(static scratch)");
+  if (rc == LR_OK) rc = launch_accept(ctx, logits, stride, drafts, cu_draft, n_branch, n_rows, n_accept, bonus, row_argmax, ptr, s);
+  if (prev_device != ctx->device) {
+    const cudaError_t e = cudaSetDevice(prev_device);
+    if (rc == LR_OK) rc = cuda_fail(e, "cudaSetDevice(restore)");
+  }
+  return rc;
 }
 
 int launch_accept(lr_ctx *ctx, const void *logits, int64_t stride, const int32_t *drafts, const int32_t *cu_draft,

@@ -1251,6 +1251,7 @@ int tc_build_host_plan(const lr_ctx *ctx, const lr_batch *b, const int32_t *req_
   }
   out.o_heads = img.add(heads.data(), heads.size() * sizeof(TcCtaHead));
   out.o_pages = img.add(pages.data(), pages.size() * sizeof(TcPage));
+  out.n_pages = (int)pages.size();
   out.o_rows = img.add(rows.data(), rows.size() * sizeof(TcRow));
   out.o_pieces = img.add(pieces.data(), pieces.size() * sizeof(TcPiece));
   out.o_cta_piece_off = img.add(cta_off.data(), cta_off.size() * sizeof(int32_t));
@@ -1266,6 +1267,12 @@ int tc_build_host_plan(const lr_ctx *ctx, const lr_batch *b, const int32_t *req_
 
 void tc_bind_device_plan(const TcHostPlan &h, unsigned char *image_base, unsigned char *scratch_base, lr_plan *p) {
   p->tc_ok = h.ok;
+  p->tc_pieces = h.n_pieces;
+  p->o_tc_pages = h.o_pages;
+  p->o_tc_heads = h.o_heads;
+  p->n_tc_pages = h.ok ? h.n_pages : 0;
+  p->n_tc_heads = h.ok ? h.n_cta : 0;
+  p->tc_partial_slots = h.n_partial_slots;
   memset(&p->tc, 0, sizeof(p->tc));
   if (!h.ok) return;
   DevTcPlan &t = p->tc;

@@ -16,7 +16,7 @@ namespace lr {
 namespace {
 
 constexpr int kThreads = 256;
-constexpr int kMaxReq = 4096;
+constexpr int kMaxReq = LR_COMMIT_MAX_REQUESTS;
 constexpr int kSmemPerReq = 7 * 4;  // bytes of shared memory per request
 
 __device__ __forceinline__ int pages_of(int n_tok) { return (n_tok + kPage - 1) / kPage; }

@@ -20,7 +20,7 @@ namespace lr {
 namespace {
 
 constexpr int kThreads = 256;
-constexpr int kMaxReq = 8192;  // the move kernels keep one prefix sum per request in shared memory
+constexpr int kMaxReq = LR_COMPACT_MAX_REQUESTS;  // the move kernels keep one prefix sum per request in shared memory
 
 __global__ void __launch_bounds__(kThreads)
 compact_scan_kernel(const int32_t *__restrict__ keep_off, const int32_t *__restrict__ keep_valid, int32_t *__restrict__ tok_off,
@@ -169,13 +169,13 @@ int launch_compact(lr_plan *p, const int32_t *keep_off, const int32_t *keep_page
   int32_t *first_moved = reinterpret_cast<int32_t *>(base + p->compact.o_first_moved);
   const int32_t *stage_off = d.compact_stage_off;  // per-request offsets into the staging area, fixed by the batch
   uint4 *staging = reinterpret_cast<uint4 *>(base + p->compact.o_staging);
-  compact_scan_kernel<<<d.n_req, kThreads, 0, s>>>(keep_off, keep_valid, tok_off, first_moved, new_len, n_pages_kept);
-  p->ctx->launches++;
-  if (int rc = cuda_fail(cudaGetLastError(), "compact_scan_kernel launch")) return rc;
   if (d.n_req > kMaxReq) {
     set_error("lr_compact: more than %d requests in one pass", kMaxReq);
     return LR_EUNSUPPORTED;
   }
+  compact_scan_kernel<<<d.n_req, kThreads, 0, s>>>(keep_off, keep_valid, tok_off, first_moved, new_len, n_pages_kept);
+  p->ctx->launches++;
+  if (int rc = cuda_fail(cudaGetLastError(), "compact_scan_kernel launch")) return rc;
   const unsigned grid = (unsigned)std::max<int64_t>(1, std::min<int64_t>((int64_t)d.n_page_slots * d.n_kv_heads, p->ctx->sm_count * 4));
   const size_t smem = sizeof(int32_t) * ((size_t)d.n_req + 1);
   compact_move_kernel<false><<<grid, kThreads, smem, s>>>(d, keep_off, keep_pages, keep_valid, tok_off, first_moved, stage_off,

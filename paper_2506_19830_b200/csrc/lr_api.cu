@@ -363,10 +363,13 @@ extern "C" int lr_plan_create(lr_ctx *ctx, const lr_batch *b, void *ws, size_t w
   if (!p) return LR_ENOMEM;
   p->ctx = ctx;
   p->pinned = nullptr;
+  p->results_pinned = nullptr;
+  p->results_pinned_cap = 0;
   p->image_bytes = L.image_bytes;
   p->workspace_d = ws;
   p->workspace_bytes = ws_bytes;
   p->attention_path = 0;
+  p->o_page_ids = L.o_page_ids;
   if (int rc = take_pinned(ctx, L.image_bytes, &p->pinned, &p->pinned_cap, &p->uploaded)) {
     delete p;
     return rc;
@@ -440,6 +443,7 @@ extern "C" int lr_plan_create(lr_ctx *ctx, const lr_batch *b, void *ws, size_t w
 extern "C" int lr_plan_destroy(lr_plan *p) {
   if (!p) return LR_OK;
   if (p->pinned) give_back_pinned(p->ctx, p->pinned, p->pinned_cap, p->uploaded);
+  if (p->results_pinned) cudaFreeHost(p->results_pinned);
   delete p;
   return LR_OK;
 }
@@ -451,6 +455,49 @@ extern "C" int lr_plan_set_attention_path(lr_plan *p, int path) {
   }
   p->attention_path = path;
   return LR_OK;
+}
+
+extern "C" int lr_plan_describe(const lr_plan *p, lr_plan_info *info) {
+  if (!p || !info) {
+    set_error("lr_plan_describe: null argument");
+    return LR_EINVAL;
+  }
+  memset(info, 0, sizeof(*info));
+  info->tensor_core_ok = p->tc_ok ? 1 : 0;
+  info->path = p->attention_path;
+  info->uses_tensor_core = (p->tc_ok && p->attention_path != 1) ? 1 : 0;
+  if (info->uses_tensor_core) {
+    info->n_cta = p->tc.n_cta;
+    info->n_pieces = p->tc_pieces;
+    info->n_merge_targets = p->tc.n_targets;
+    info->n_partial_slots = p->tc_partial_slots;
+  }
+  return LR_OK;
+}
+
+extern "C" int lr_plan_debug_set_page(lr_plan *p, int32_t page_slot, int32_t new_id, void *stream) {
+  if (!p || page_slot < 0 || page_slot >= p->dev.n_page_slots) {
+    set_error("lr_plan_debug_set_page: bad argument");
+    return LR_EINVAL;
+  }
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  // the pinned image is the source of the last upload: wait until that copy has read it
+  if (int rc = cuda_fail(cudaEventSynchronize(p->uploaded), "cudaEventSynchronize(plan image)")) return rc;
+  unsigned char *img = reinterpret_cast<unsigned char *>(p->pinned);
+  int32_t *ids = reinterpret_cast<int32_t *>(img + p->o_page_ids);
+  const int32_t old_id = ids[page_slot];
+  ids[page_slot] = new_id;
+  // physical page ids are distinct within a batch, so the old id names this slot in the attention tables too
+  TcPage *pages = reinterpret_cast<TcPage *>(img + p->o_tc_pages);
+  for (int i = 0; i < p->n_tc_pages; ++i)
+    if (pages[i].page == old_id && (pages[i].meta & 31u) != 0u) pages[i].page = new_id;
+  TcCtaHead *heads = reinterpret_cast<TcCtaHead *>(img + p->o_tc_heads);
+  for (int c = 0; c < p->n_tc_heads; ++c)
+    for (int k = 0; k < 32; ++k)
+      if (heads[c].first_pages[k] == old_id && heads[c].piece1 > heads[c].piece0) heads[c].first_pages[k] = new_id;
+  cudaError_t e = cudaMemcpyAsync(p->workspace_d, p->pinned, p->image_bytes, cudaMemcpyHostToDevice, s);
+  if (e == cudaSuccess) e = cudaEventRecord(p->uploaded, s);
+  return cuda_fail(e, "lr_plan_debug_set_page upload");
 }
 
 // ---- steps ---------------------------------------------------------------------
@@ -704,8 +751,23 @@ extern "C" int lr_verify_pass_host(lr_plan *p, const lr_pass_host_io *io, const 
   if (int rc = lr_commit(p, b + L.verdict, I(L.n_accept), I(L.n_steps), I(L.survivor), I(L.committed), I(L.keep_off),
                          I(L.keep_pages), I(L.keep_valid), I(L.free_off), I(L.free_pages), stream))
     return rc;
+  // Results: the attention output goes straight to its host buffer; the ten integer arrays lie next to one another in
+  // the staging buffer and leave in one copy, through a pinned buffer the plan keeps, then to the caller's arrays.
+  e = cudaMemcpyAsync(io->out_h, b + L.out, qo, cudaMemcpyDeviceToHost, s);
+  if (e != cudaSuccess) return cuda_fail(e, "lr_verify_pass_host: device-to-host copy of the output");
+  const size_t small_bytes = L.scratch - L.n_accept;
+  if (p->results_pinned_cap < small_bytes) {
+    if (p->results_pinned) cudaFreeHost(p->results_pinned);
+    p->results_pinned = nullptr;
+    p->results_pinned_cap = 0;
+    if (int rc = cuda_fail(cudaMallocHost(&p->results_pinned, small_bytes), "cudaMallocHost(pass results)")) return rc;
+    p->results_pinned_cap = small_bytes;
+  }
+  e = cudaMemcpyAsync(p->results_pinned, b + L.n_accept, small_bytes, cudaMemcpyDeviceToHost, s);
+  if (e != cudaSuccess) return cuda_fail(e, "lr_verify_pass_host: device-to-host copy of the integer results");
+  const int rc = lr_poll_status(p, stream, nullptr);  // waits for the stream
+  if (rc != LR_OK && rc != LR_ETIMEOUT && rc != LR_EBOUNDS) return rc;
   struct Back { void *dst; size_t off, n; } back[] = {
-      {io->out_h, L.out, qo},
       {io->n_accept_h, L.n_accept, (size_t)d.n_branch * 4},
       {io->bonus_id_h, L.bonus, (size_t)d.n_branch * 4},
       {io->n_steps_accepted_h, L.n_steps, (size_t)d.n_req * 4},
@@ -717,11 +779,8 @@ extern "C" int lr_verify_pass_host(lr_plan *p, const lr_pass_host_io *io, const 
       {io->keep_valid_h, L.keep_valid, (size_t)d.n_page_slots * 4},
       {io->free_pages_h, L.free_pages, (size_t)d.n_page_slots * 4},
   };
-  for (const Back &k : back) {
-    e = cudaMemcpyAsync(k.dst, b + k.off, k.n, cudaMemcpyDeviceToHost, s);
-    if (e != cudaSuccess) return cuda_fail(e, "lr_verify_pass_host: device-to-host copies");
-  }
-  return lr_poll_status(p, stream, nullptr);
+  for (const Back &k : back) memcpy(k.dst, reinterpret_cast<unsigned char *>(p->results_pinned) + (k.off - L.n_accept), k.n);
+  return rc;
 }
 
 extern "C" const char *lr_strerror(int st) {

@@ -130,9 +130,15 @@ struct lr_plan {
   lr::DevTcPlan tc;
   bool tc_ok;             // shape allows the tensor-core path
   int attention_path;     // 0 auto, 1 generic, 2 tensor core
+  int tc_pieces, tc_partial_slots;  // for lr_plan_describe
+  // where the physical page ids sit in the image (lr_plan_debug_set_page)
+  size_t o_page_ids, o_tc_pages, o_tc_heads;
+  int n_tc_pages, n_tc_heads;
   std::vector<unsigned char> staging;  // host copy of the uploaded image (kept alive for the async copy)
   void *pinned;           // pinned host image
   size_t pinned_cap;
+  void *results_pinned;   // pinned bounce buffer for the integer results of lr_verify_pass_host (allocated on first use)
+  size_t results_pinned_cap;
   cudaEvent_t uploaded;   // recorded after the image's upload
   size_t image_bytes;
   void *workspace_d;
@@ -160,7 +166,7 @@ struct Image {
 struct TcHostPlan {
   bool ok = false;  // shape supported by the tensor-core path
   size_t o_heads = 0, o_pages = 0, o_rows = 0, o_pieces = 0, o_cta_piece_off = 0, o_reqs = 0, o_targets = 0;  // image offsets
-  int n_cta = 0, n_targets = 0, n_pieces = 0, n_partial_slots = 0, tokens_per_mtile = 0;
+  int n_cta = 0, n_targets = 0, n_pieces = 0, n_partial_slots = 0, tokens_per_mtile = 0, n_pages = 0;
   // scratch region behind the image: (exponent, sum) pairs, then fp32 partial outputs
   size_t s_ml = 0, s_o = 0, scratch_bytes = 0, scratch_zero_bytes = 0;
 };

@@ -6,7 +6,7 @@ import pytest
 from lr_workloads import Model, bf16_to_f32, build_batch, fill_kv, fill_logits_and_drafts, fill_q, fill_verdicts
 from oracle import lr_oracle as O
 from paper_2506_19830_b200.cycle import BranchInput, PagedCycleEngine, RequestInput
-from gpu_util import MAX_ABS, MAX_REL_LARGE, MEAN_ABS
+from gpu_util import REL_LARGE, assert_attention_close
 
 pytestmark = pytest.mark.gpu
 PAGE = 16
@@ -71,7 +71,7 @@ def test_cycles_keep_the_cache_equal_to_the_logical_sequences(head_dim, tree):
         for key in ("n_accept", "bonus_id", "n_steps_accepted", "survivor", "committed_len"):
             assert np.array_equal(got[key], ref[key]), (cycle, key)
         err = np.abs(bf16_to_f32(got["out"]).astype(np.float64) - ref["out"])
-        assert (err <= np.maximum(MAX_ABS, MAX_REL_LARGE * np.abs(ref["out"]))).all() and err.mean() <= MEAN_ABS, (cycle, err.max(), err.mean())
+        assert_attention_close(err, ref["out"], REL_LARGE)  # random ragged cycles: the random generators' bound
         # grow the logical sequences by what was committed, token by token from the oracle's cache
         for r in range(n_req):
             s0 = int(b.req_span_off[r])

@@ -9,7 +9,7 @@ from lr_workloads import Model, build_batch, make_config, make_random_small, mak
 from oracle import lr_oracle as O
 from paper_2506_19830_b200 import binding as B
 from paper_2506_19830_b200 import runner as R
-from gpu_util import check_commit, run_and_check_pass
+from gpu_util import REL_LARGE, attention_path_for, check_commit, run_and_check_pass
 
 pytestmark = pytest.mark.gpu
 
@@ -20,25 +20,25 @@ def _rng(seed):
 
 @pytest.mark.parametrize("seed", list(range(12)))
 def test_whole_pass_random_trees(seed):
-    run_and_check_pass(make_random_tree(500 + seed))
+    run_and_check_pass(make_random_tree(500 + seed), rel_large=REL_LARGE)
 
 
 @pytest.mark.parametrize("seed", list(range(4)))
 def test_whole_pass_random_trees_tensor_core_path(seed):
-    run_and_check_pass(make_random_tree(600 + seed, head_dim=128))
+    run_and_check_pass(make_random_tree(600 + seed, head_dim=128), rel_large=REL_LARGE)
 
 
 def test_many_small_passes_on_the_tensor_core_path():
     """Tiny passes put several one-tile pieces into one CTA, where one of its two streams has nothing to do: the
     piece-by-piece barrier phases must still line up (seed 5000 once ran into an expired wait)."""
     for seed in [5000] + list(range(5100, 5140)):
-        run_and_check_pass(make_random_tree(seed, head_dim=128))
-        run_and_check_pass(make_random_small(seed, head_dim=128))
+        run_and_check_pass(make_random_tree(seed, head_dim=128), rel_large=REL_LARGE)
+        run_and_check_pass(make_random_small(seed, head_dim=128), rel_large=REL_LARGE)
 
 
 @pytest.mark.parametrize("seed", list(range(4)))
 def test_whole_pass_random_trees_generic_path(seed):
-    run_and_check_pass(make_random_tree(700 + seed), path=B.PATH_GENERIC)
+    run_and_check_pass(make_random_tree(700 + seed), path=B.PATH_GENERIC, rel_large=REL_LARGE)
 
 
 @pytest.mark.parametrize("W,gamma,size", [(2, 2, "tiny"), (3, 2, "tiny"), (2, 3, "layer"), (4, 2, "layer"), (2, 2, "serving")])
@@ -55,6 +55,7 @@ def test_a_chain_written_with_parents_gives_the_same_bits(make):
     for batch in (b, dataclasses.replace(b, seg_parent=parent)):
         ctx = B.Context(batch.model, 0)
         plan = B.Plan(ctx, batch)
+        plan.lr_plan_set_attention_path(attention_path_for(batch.model))
         x, y = R.DeviceInputs(batch, t), R.PassOutputs(batch)
         R.run_pass(ctx, plan, x, y)
         assert plan.lr_poll_status() == 0

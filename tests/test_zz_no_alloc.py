@@ -1,6 +1,7 @@
 """``lr_accept_greedy_static`` -- greedy acceptance for callers that cannot hand the library a
 scratch buffer (an engine whose HBM is fully committed to its KV cache, or code that must not call
-cudaMalloc because it stalls the device) -- must give exactly what ``lr_accept_greedy`` gives.
+cudaMalloc because it stalls the device) -- must give exactly what ``lr_accept_greedy`` gives, and
+what the CPU oracle's acceptance rule gives.
 
 This file sorts last on purpose: a run that stops at the first failure has then already executed
 every other test.  It passes on its own in a fresh process and after the rest of the suite.
@@ -10,6 +11,7 @@ import pytest
 import torch
 
 from lr_workloads import make_config, make_random_small
+from oracle import lr_oracle as O
 from paper_2506_19830_b200 import binding as B
 from paper_2506_19830_b200 import runner as R
 
@@ -25,12 +27,15 @@ def _both(w, dev="cuda:0"):
     ref = [torch.empty(b.n_branch, **i32), torch.empty(b.n_branch, **i32), torch.empty(n_rows, **i32)]
     ctx.lr_accept_greedy(x.logits, x.draft_ids, x.cu_draft, ref[0], ref[1], B.Context.accept_scratch(n_rows, dev), ref[2])
     torch.cuda.synchronize()
+    n_ref, bonus_ref, arg_ref = O.accept_greedy(t.logits, t.draft_ids, b.cu_draft)
+    oracle = [torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).to(dev) for a in (n_ref, bonus_ref, arg_ref)]
     for call in range(2):  # two calls in a row: the second one sees whatever the first left in the array
         got = [torch.full((b.n_branch,), -7, **i32), torch.full((b.n_branch,), -7, **i32), torch.full((n_rows,), -7, **i32)]
         ctx.lr_accept_greedy_static(x.logits, x.draft_ids, x.cu_draft, got[0], got[1], got[2])
         torch.cuda.synchronize()
-        for name, g, r in zip(("n_accept", "bonus_id", "row_argmax"), got, ref):
+        for name, g, r, o in zip(("n_accept", "bonus_id", "row_argmax"), got, ref, oracle):
             assert torch.equal(g, r), f"call {call}: {name} differs from lr_accept_greedy"  # integer results: bit-exact
+            assert torch.equal(g, o), f"call {call}: {name} differs from the oracle"
     ctx.close()
 
 
