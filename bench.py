@@ -425,7 +425,9 @@ class Measurement:
         uses_tc = bool(self.info["uses_tensor_core"])
         plain = self.args.path == 0 and not self.args.carry_in
         timed = "attn_generic_kernel"
-        if uses_tc:
+        if uses_tc and self.info["path"] == 3:
+            timed = "attn_pair_kernel"
+        elif uses_tc:
             timed = "attn_tc_kernel" + (" + attn_tc_merge_kernel" if self.info["n_merge_targets"] > 0 and TC_MERGE_IS_A_LAUNCH else "")
         roof.update({"traffic": _traffic_for(self.label, uses_tc) if plain else None, "kernel": "lr_verify_attention",
                      "kernel_us": kernel_us["attention"], "algorithmic_bytes": a_bytes, "algorithmic_flops": a_flops,

@@ -21,7 +21,7 @@ LR_OK = 0
 STATUS_NAMES = {0: "LR_OK", -1: "LR_EINVAL", -2: "LR_EUNSUPPORTED", -3: "LR_ECUDA", -4: "LR_ETIMEOUT", -5: "LR_EBOUNDS",
                 -6: "LR_ENOMEM"}
 
-PATH_AUTO, PATH_GENERIC, PATH_TENSOR_CORE = 0, 1, 2
+PATH_AUTO, PATH_GENERIC, PATH_TENSOR_CORE, PATH_PAIR = 0, 1, 2, 3
 ACCEPT_STATIC_MAX_ROWS = 4096  # LR_ACCEPT_STATIC_MAX_ROWS
 COMMIT_MAX_REQUESTS = 4096  # LR_COMMIT_MAX_REQUESTS
 COMPACT_MAX_REQUESTS = 8192  # LR_COMPACT_MAX_REQUESTS

@@ -113,7 +113,8 @@ struct Layout {
   size_t compact_tokens;
   std::vector<int32_t> cu_draft;
   TcHostPlan tc;
-  size_t image_bytes, total_bytes;
+  PairHostPlan pr;
+  size_t image_bytes, total_bytes, pair_scratch_off;
 };
 
 static int build_layout(const lr_ctx *ctx, const lr_batch *b, Layout &L) {
@@ -216,8 +217,10 @@ static int build_layout(const lr_ctx *ctx, const lr_batch *b, Layout &L) {
   L.o_status = g.add(zero2, sizeof(zero2));
   L.cu_draft = cu_draft;
   if (int rc = tc_build_host_plan(ctx, b, req_br_off.data(), span_tin.data(), span_last.data(), L.tc, g)) return rc;
+  if (int rc = pair_build_host_plan(ctx, b, req_br_off.data(), span_tin.data(), span_last.data(), L.pr, g)) return rc;
   L.image_bytes = align_up(g.bytes.size(), 256);
-  L.total_bytes = L.image_bytes + align_up(L.tc.scratch_bytes, 256);
+  L.pair_scratch_off = L.image_bytes + align_up(L.tc.scratch_bytes, 256);
+  L.total_bytes = L.pair_scratch_off + align_up(L.pr.scratch_bytes, 256);
   return LR_OK;
 }
 
@@ -278,6 +281,7 @@ extern "C" int lr_create(lr_ctx **out, const lr_model *m, int device) {
   c->tmap_encode = nullptr;
   if (int rc = init_commit_kernel()) { delete c; return rc; }
   if (int rc = init_attn_tc_kernel()) { delete c; return rc; }
+  if (int rc = init_attn_pair_kernel()) { delete c; return rc; }
   *out = c;
   return LR_OK;
 }
@@ -426,10 +430,13 @@ extern "C" int lr_plan_create(lr_ctx *ctx, const lr_batch *b, void *ws, size_t w
   p->n_rows_logits = p->n_drafts + b->n_branch;
   p->n_verdicts = b->n_span - b->n_req;
   tc_bind_device_plan(L.tc, base, base + L.image_bytes, p);
+  pair_bind_device_plan(L.pr, base, base + L.pair_scratch_off, p);
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
   cudaError_t e = cudaMemcpyAsync(ws, p->pinned, L.image_bytes, cudaMemcpyHostToDevice, s);
   if (e == cudaSuccess && L.tc.scratch_zero_bytes)
     e = cudaMemsetAsync(base + L.image_bytes, 0, L.tc.scratch_zero_bytes, s);
+  if (e == cudaSuccess && L.pr.scratch_zero_bytes)
+    e = cudaMemsetAsync(base + L.pair_scratch_off, 0, L.pr.scratch_zero_bytes, s);
   if (e == cudaSuccess) e = cudaEventRecord(p->uploaded, s);
   if (e != cudaSuccess) {
     give_back_pinned(ctx, p->pinned, p->pinned_cap, p->uploaded);
@@ -449,7 +456,7 @@ extern "C" int lr_plan_destroy(lr_plan *p) {
 }
 
 extern "C" int lr_plan_set_attention_path(lr_plan *p, int path) {
-  if (!p || path < 0 || path > 2) {
+  if (!p || path < 0 || path > 3) {
     set_error("lr_plan_set_attention_path: bad argument");
     return LR_EINVAL;
   }
@@ -465,6 +472,16 @@ extern "C" int lr_plan_describe(const lr_plan *p, lr_plan_info *info) {
   memset(info, 0, sizeof(*info));
   info->tensor_core_ok = p->tc_ok ? 1 : 0;
   info->path = p->attention_path;
+  if (p->attention_path == 3) {
+    info->uses_tensor_core = p->pair_ok ? 1 : 0;
+    if (p->pair_ok) {
+      info->n_cta = 2 * p->pr.n_pairs;
+      info->n_pieces = p->pr_pieces;
+      info->n_merge_targets = p->pr.n_targets;
+      info->n_partial_slots = p->pr_partial_slots;
+    }
+    return LR_OK;
+  }
   info->uses_tensor_core = (p->tc_ok && p->attention_path != 1) ? 1 : 0;
   if (info->uses_tensor_core) {
     info->n_cta = p->tc.n_cta;
@@ -495,6 +512,13 @@ extern "C" int lr_plan_debug_set_page(lr_plan *p, int32_t page_slot, int32_t new
   for (int c = 0; c < p->n_tc_heads; ++c)
     for (int k = 0; k < 32; ++k)
       if (heads[c].first_pages[k] == old_id && heads[c].piece1 > heads[c].piece0) heads[c].first_pages[k] = new_id;
+  TcPage *ppages = reinterpret_cast<TcPage *>(img + p->o_pr_pages);
+  for (int i = 0; i < p->n_pr_pages; ++i)
+    if (ppages[i].page == old_id && (ppages[i].meta & 31u) != 0u) ppages[i].page = new_id;
+  PrHead *pheads = reinterpret_cast<PrHead *>(img + p->o_pr_heads);
+  for (int c = 0; c < p->n_pr_heads; ++c)
+    for (int k = 0; k < 32; ++k)
+      if (pheads[c].first_pages[k] == old_id && pheads[c].piece1 > pheads[c].piece0) pheads[c].first_pages[k] = new_id;
   cudaError_t e = cudaMemcpyAsync(p->workspace_d, p->pinned, p->image_bytes, cudaMemcpyHostToDevice, s);
   if (e == cudaSuccess) e = cudaEventRecord(p->uploaded, s);
   return cuda_fail(e, "lr_plan_debug_set_page upload");
@@ -513,6 +537,13 @@ extern "C" int lr_verify_attention(lr_plan *p, const void *q, const void *k, con
   }
   if (!(scale > 0.f)) scale = 1.0f / sqrtf((float)p->dev.head_dim);
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  if (p->attention_path == 3) {
+    if (!p->pair_ok) {
+      set_error("lr_verify_attention: the CTA-pair tensor-core path does not support this shape");
+      return LR_EUNSUPPORTED;
+    }
+    return launch_attn_pair(p, q, k, v, out, lse, scale, s);
+  }
   bool use_tc = p->attention_path == 2 || (p->attention_path == 0 && p->tc_ok);
   if (use_tc) {
     if (!p->tc_ok) {

@@ -108,6 +108,40 @@ struct DevTcPlan {
   float *partial_ml;         // [n_slots][128][2] (reference exponent in log2 units, sum)
 };
 
+// ---- CTA-pair attention plan (device side) -----------------------------------
+// Two CTAs on neighbouring SMs work as one unit: CTA c of the pair owns M-tile mtile0 + c of a piece (its query
+// rows, scores, probabilities and output accumulator) and supplies half of every KV tile; one tcgen05.mma with
+// cta_group::2 (M = 256) applies the whole tile to both M-tiles.  Pages, rows and requests are described as for the
+// single-CTA plan above.
+struct PrPiece {
+  int32_t req, kv_head;
+  int32_t mtile0, n_mt;           // first M-tile and how many (1 or 2: with 1 the second CTA only lends its half of the KV tile)
+  int32_t tile_begin, tile_end;   // tiles of the request's extended chain
+  int32_t slot[2];                // per CTA of the pair: >= 0 partial slot, -1 write the final output, -2 nothing to write
+  int32_t target[2];              // per CTA: merge target (index into targets / counters), -1 when slot < 0
+};
+struct PrHead {                   // everything a pair needs to start, in one 256-byte record
+  int32_t piece0, piece1;
+  PrPiece first;
+  TcReq first_req;
+  int32_t first_pages[32];        // physical ids of pages 32*c .. 32*c+31 of that request, c = first.tile_begin / 4; -1 = absent
+  int32_t pad[12];
+};
+struct DevPairPlan {
+  const PrHead *heads;            // [n_pairs]
+  const TcPage *pages;
+  const TcRow *rows;
+  const PrPiece *pieces;
+  const TcReq *reqs;
+  const TcTarget *targets;
+  int32_t n_pairs, n_targets;
+  int32_t tokens_per_mtile;
+  uint32_t wait_limit_us;         // bound of every device-side wait (test hook: lr_plan_debug_set_wait_limit)
+  float *partial_o;               // [n_slots][32 chunks of 4 channels][128 rows][4] fp32, unnormalised
+  float *partial_ml;              // [n_slots][128][2] (reference exponent in log2 units, sum)
+  uint32_t *counters;             // [n_targets] arrival tickets of the contributors of a target; zero between launches
+};
+
 }  // namespace lr
 
 struct lr_ctx {
@@ -128,8 +162,13 @@ struct lr_plan {
   lr_ctx *ctx;
   lr::DevBatch dev;
   lr::DevTcPlan tc;
+  lr::DevPairPlan pr;
   bool tc_ok;             // shape allows the tensor-core path
-  int attention_path;     // 0 auto, 1 generic, 2 tensor core
+  bool pair_ok;           // shape allows the CTA-pair tensor-core path
+  int pr_pieces, pr_partial_slots;
+  size_t o_pr_pages, o_pr_heads;
+  int n_pr_pages, n_pr_heads;
+  int attention_path;     // 0 auto, 1 generic, 2 tensor core (single CTA), 3 tensor core (CTA pairs)
   int tc_pieces, tc_partial_slots;  // for lr_plan_describe
   // where the physical page ids sit in the image (lr_plan_debug_set_page)
   size_t o_page_ids, o_tc_pages, o_tc_heads;
@@ -175,6 +214,18 @@ int tc_build_host_plan(const lr_ctx *ctx, const lr_batch *b, const int32_t *req_
                        const int32_t *span_last, TcHostPlan &out, Image &img);
 void tc_bind_device_plan(const TcHostPlan &h, unsigned char *image_base, unsigned char *scratch_base, lr_plan *p);
 
+// Host-side result of planning the CTA-pair attention for one batch.
+struct PairHostPlan {
+  bool ok = false;
+  size_t o_heads = 0, o_pages = 0, o_rows = 0, o_pieces = 0, o_reqs = 0, o_targets = 0;  // image offsets
+  int n_pairs = 0, n_targets = 0, n_pieces = 0, n_partial_slots = 0, tokens_per_mtile = 0, n_pages = 0;
+  // scratch region behind the image: ticket counters, (exponent, sum) pairs, fp32 partial outputs
+  size_t s_counters = 0, s_ml = 0, s_o = 0, scratch_bytes = 0, scratch_zero_bytes = 0;
+};
+int pair_build_host_plan(const lr_ctx *ctx, const lr_batch *b, const int32_t *req_br_off, const int32_t *span_tin,
+                         const int32_t *span_last, PairHostPlan &out, Image &img);
+void pair_bind_device_plan(const PairHostPlan &h, unsigned char *image_base, unsigned char *scratch_base, lr_plan *p);
+
 void set_error(const char *fmt, ...);
 
 // Launch as a programmatic dependent of the kernel before it in the stream: the grid is set up while that kernel
@@ -199,6 +250,9 @@ int cuda_fail(cudaError_t e, const char *what);
 int init_kernels(lr_ctx *ctx);  // per-device function attributes; called by lr_create
 int init_commit_kernel();
 int init_attn_tc_kernel();
+int init_attn_pair_kernel();
+int launch_attn_pair(lr_plan *p, const void *q, const void *k, const void *v, void *out, float *lse, float scale,
+                     cudaStream_t s);
 int launch_attn_generic(lr_plan *p, const void *q, const void *k, const void *v, void *out, float *lse, float scale,
                         cudaStream_t s);
 int launch_attn_tc(lr_plan *p, const void *q, const void *k, const void *v, void *out, float *lse, float scale,

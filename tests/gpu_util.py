@@ -69,7 +69,7 @@ def run_and_check_pass(w, path=None, check_rows_of_branches=None, rel_large: flo
         path = attention_path_for(b.model)
     plan.lr_plan_set_attention_path(path)
     info = plan.lr_plan_describe()
-    assert info["uses_tensor_core"] == (1 if path == B.PATH_TENSOR_CORE else 0), info
+    assert info["uses_tensor_core"] == (1 if path in (B.PATH_TENSOR_CORE, B.PATH_PAIR) else 0), info
     x = R.DeviceInputs(b, t)
     y = R.PassOutputs(b)
     y.out.fill_(float("nan"))
