@@ -191,6 +191,19 @@ int lr_plan_set_attention_path(lr_plan *plan, int path);
  * (lr_poll_status); it never dereferences the id. */
 int lr_plan_debug_set_page(lr_plan *plan, int32_t page_slot, int32_t new_id, void *stream);
 
+/* Test hook for the bounded device-side waits: every wait of the tensor-core attention kernels of later
+ * lr_verify_attention calls on this plan gives up after `microseconds` (default: one second).  With a limit
+ * shorter than a trip to memory a wait expires while its data is still on the way; the CTA then records
+ * LR_ETIMEOUT in the status word, lets the copies and products it has in flight finish (bounded again), releases
+ * its tensor memory and returns.  The output of such a pass is unspecified; the context stays usable. */
+int lr_plan_debug_set_wait_limit(lr_plan *plan, uint32_t microseconds);
+
+/* Test hook that makes one wait run out: the first CTA of the tensor-core attention kernels expects `bytes` more on
+ * its first KV stage than its copies deliver, so the barrier of that stage never completes and the waits on it
+ * expire after the limit above -- LR_ETIMEOUT through lr_poll_status, nothing worse: the CTA leaves through its
+ * abort path, every other CTA finishes normally.  0 switches the hook off.  Set a short limit first. */
+int lr_plan_debug_set_phantom_bytes(lr_plan *plan, uint32_t bytes);
+
 /* Bytes of scratch lr_accept_greedy needs for n_rows logits rows.  The scratch
  * must be zero-filled before its first use; every call leaves it zero-filled. */
 int lr_accept_scratch_bytes(int32_t n_rows, size_t *bytes_out);

@@ -86,6 +86,8 @@ def lib() -> C.CDLL:
             "lr_plan_set_attention_path": [vp, C.c_int],
             "lr_plan_describe": [vp, C.POINTER(lr_plan_info)],
             "lr_plan_debug_set_page": [vp, i32, i32, vp],
+            "lr_plan_debug_set_wait_limit": [vp, C.c_uint32],
+            "lr_plan_debug_set_phantom_bytes": [vp, C.c_uint32],
             "lr_verify_attention": [vp, vp, vp, vp, vp, vp, f32, vp],
             "lr_accept_scratch_bytes": [i32, C.POINTER(sz)],
             "lr_accept_greedy": [vp, vp, i64, vp, vp, i32, i32, vp, vp, vp, vp, vp],
@@ -277,6 +279,12 @@ class Plan:
 
     def lr_plan_debug_set_page(self, page_slot: int, new_id: int, stream=None) -> None:
         _check(lib().lr_plan_debug_set_page(self.handle, page_slot, new_id, _stream_ptr(stream)), "lr_plan_debug_set_page")
+
+    def lr_plan_debug_set_wait_limit(self, microseconds: int) -> None:
+        _check(lib().lr_plan_debug_set_wait_limit(self.handle, microseconds), "lr_plan_debug_set_wait_limit")
+
+    def lr_plan_debug_set_phantom_bytes(self, n_bytes: int) -> None:
+        _check(lib().lr_plan_debug_set_phantom_bytes(self.handle, n_bytes), "lr_plan_debug_set_phantom_bytes")
 
     def lr_plan_describe(self) -> dict:
         info = lr_plan_info()

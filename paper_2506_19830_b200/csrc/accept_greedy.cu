@@ -189,34 +189,37 @@ accept_greedy_kernel(const uint16_t *__restrict__ logits, int64_t row_stride, in
   // ---- last CTA: per-branch longest matching prefix + bonus ------------------
   __threadfence();
   volatile unsigned long long *vk = row_key;
-  // One warp per branch: the L + 1 rows of a branch are loaded 32 at a time, all at once, and the first
-  // mismatch is found with a ballot -- no chain of dependent loads along the drafts.
-  const int lane = tid & 31;
-  for (int b = tid >> 5; b < n_branch; b += kThreads / 32) {
+  // One thread per branch, so that hundreds of branches cost one pass: the bounds of its draft range with two loads in
+  // flight, then its rows eight at a time -- keys and drafts of a chunk are loaded together, so a chunk costs one
+  // round trip to L2 whatever the branch count -- and the scan stops at the first mismatch.
+  for (int b = tid; b < n_branch; b += kThreads) {
     const int32_t d0 = cu_draft[b], L = cu_draft[b + 1] - d0;
     const int32_t r0 = d0 + b;
     int32_t n = L, bonus = 0;
     bool found = false;
-    for (int32_t i0 = 0; i0 <= L && !found; i0 += 32) {
-      const int32_t i = i0 + lane;
-      int32_t t = 0;
-      bool mismatch = false;
-      if (i <= L) {
-        t = (int32_t)(0xFFFFFFFFu - (uint32_t)(vk[r0 + i] & 0xFFFFFFFFull));
-        mismatch = (i == L) || (draft_ids[d0 + i] != t);  // row L has no draft: the scan always stops there
+    for (int32_t i0 = 0; i0 <= L && !found; i0 += 8) {
+      int32_t t[8], dr[8];
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        const int32_t i = i0 + k;
+        t[k] = 0;
+        dr[k] = -1;
+        if (i <= L) t[k] = (int32_t)(0xFFFFFFFFu - (uint32_t)(vk[r0 + i] & 0xFFFFFFFFull));
+        if (i < L) dr[k] = draft_ids[d0 + i];
       }
-      const unsigned m = __ballot_sync(0xFFFFFFFFu, mismatch);
-      if (m != 0u) {
-        const int first = __ffs(m) - 1;
-        n = i0 + first;
-        bonus = __shfl_sync(0xFFFFFFFFu, t, first);
-        found = true;
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        const int32_t i = i0 + k;
+        // row L has no draft: the scan always stops there
+        if (!found && i <= L && (i == L || dr[k] != t[k])) {
+          found = true;
+          n = i;
+          bonus = t[k];
+        }
       }
     }
-    if (lane == 0) {
-      n_accept[b] = n;
-      bonus_id[b] = bonus;
-    }
+    n_accept[b] = n;
+    bonus_id[b] = bonus;
   }
   if (row_argmax != nullptr)
     for (int r = tid; r < n_rows; r += kThreads)

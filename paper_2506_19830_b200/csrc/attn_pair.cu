@@ -636,7 +636,8 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constan
         ok = wait_bar_warp(&ctrl->kv_empty[stage], ((ring / kStages) & 1u) ^ 1u, wc, 210);
         if (!ok) break;
         if (lane == 0) {
-          const uint32_t bytes = (uint32_t)mine_k * 4096u + (uint32_t)v_in_tile * 2048u;
+          const uint32_t bytes = (uint32_t)mine_k * 4096u + (uint32_t)v_in_tile * 2048u +
+                                 ((pair == 0 && cta == 0 && ring == 0) ? pp.phantom_tx_bytes : 0u);
           if (bytes > 0) mbar_arrive_expect_tx(&ctrl->kv_full[stage], bytes);
           else mbar_arrive(&ctrl->kv_full[stage]);
         }
@@ -940,11 +941,11 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constan
         }
         const TcTarget tg = pp.targets[target];
         bar_sync_softmax();
-        const bool last = ok && *reinterpret_cast<volatile uint32_t *>(&ctrl->ticket) == (uint32_t)tg.n_slots - 1u;
+        const bool last = *reinterpret_cast<volatile uint32_t *>(&ctrl->ticket) == (uint32_t)tg.n_slots - 1u;
         bar_sync_softmax();  // everybody has read the ticket before the next piece may overwrite it
         if (last) {
-          merge_row(tg.slot_begin, tg.n_slots, r, g, ri.q_index, out, lse, pp.partial_o, pp.partial_ml);
-          if (threadIdx.x == 0) pp.counters[target] = 0u;  // ready for the next launch
+          if (ok) merge_row(tg.slot_begin, tg.n_slots, r, g, ri.q_index, out, lse, pp.partial_o, pp.partial_ml);
+          if (threadIdx.x == 0) pp.counters[target] = 0u;  // ready for the next launch, also after an aborted pass
         }
       }
     }
@@ -1238,6 +1239,7 @@ void pair_bind_device_plan(const PairHostPlan &h, unsigned char *image_base, uns
   t.n_targets = h.n_targets;
   t.tokens_per_mtile = h.tokens_per_mtile;
   t.wait_limit_us = 1000000u;  // one second per wait, measured on the global timer
+  t.phantom_tx_bytes = 0;
   t.counters = reinterpret_cast<uint32_t *>(scratch_base + h.s_counters);
   t.partial_ml = reinterpret_cast<float *>(scratch_base + h.s_ml);
   t.partial_o = reinterpret_cast<float *>(scratch_base + h.s_o);

@@ -81,7 +81,6 @@ constexpr int kAtomBytes = 1024;   // K/V tiles: 8 keys x 64 channels, one 128-b
 constexpr int kGroupBytes = 2048;  // ... two atoms (the two channel halves) per 8-key group
 constexpr int kThreads = 384;
 constexpr int kPagesPerTile = 8;
-constexpr uint64_t kWaitLimitNs = 1000ull * 1000ull * 1000ull;  // one second per wait, measured on the global timer
 constexpr uint64_t kDrainLimitNs = 50ull * 1000ull * 1000ull;
 constexpr float kRescaleThreshold = 8.0f;  // log2 units: the reference exponent follows the row maximum within 2^8
 constexpr float kRedoThreshold = 64.0f;    // log2 units: beyond this a tile is redone with its own maximum as reference
@@ -94,6 +93,7 @@ struct __align__(8) Ctrl {
   uint64_t xch;           // stream 1 -> stream 0: its (m, l) are published and its accumulator is final
   uint32_t tmem_base;
   int abort_flag;
+  uint64_t wait_limit_ns;  // bound of every wait, measured on the global timer
   float2 ml_xch[128];     // (reference exponent, row sum) of stream 1's rows, for the in-CTA combination
 };
 constexpr int kCtrlBytes = 2048;
@@ -257,20 +257,26 @@ __device__ __forceinline__ uint64_t global_ns() {
 
 // Bounded wait: gives up after kWaitLimitNs of wall time.  Returns false when the wait expired or
 // another role of the CTA gave up.
-__device__ __forceinline__ bool wait_bar(uint64_t *bar, uint32_t parity, Ctrl *ctrl, int32_t *status, int code) {
+__device__ __forceinline__ bool wait_bar_lane(uint64_t *bar, uint32_t parity, Ctrl *ctrl, int32_t *status, int code) {
   if (mbar_test_wait(bar, parity)) return true;
   const uint64_t t0 = global_ns();
   for (uint32_t i = 1;; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((i & 31u) == 0u) {
       if (*reinterpret_cast<volatile int *>(&ctrl->abort_flag)) return false;
-      if (global_ns() - t0 > kWaitLimitNs) break;
+      if (global_ns() - t0 > ctrl->wait_limit_ns) break;
     }
   }
   *reinterpret_cast<volatile int *>(&ctrl->abort_flag) = 1;
   status[0] = kDevTimeout;
   status[1] = code;
   return false;
+}
+
+// Every wait of the kernel is made by a whole warp: the warp goes on only if every lane's wait succeeded, so that it
+// never executes its warp-wide instructions half in and half out of an abort.
+__device__ __forceinline__ bool wait_bar(uint64_t *bar, uint32_t parity, Ctrl *ctrl, int32_t *status, int code) {
+  return __all_sync(0xFFFFFFFFu, wait_bar_lane(bar, parity, ctrl, status, code)) != 0;
 }
 
 // ---- ring order ----------------------------------------------------------------------
@@ -505,6 +511,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant_
     mbar_init(&ctrl->epi_done, 256);
     mbar_init(&ctrl->xch, 128);
     ctrl->abort_flag = 0;
+    ctrl->wait_limit_ns = (uint64_t)tc.wait_limit_us * 1000ull;
     fence_barrier_init();
   }
   if (warp == 9) {
@@ -568,7 +575,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant_
       int32_t pg_nxt = load_chunk(c_cur + 1), pg_cur;
       if (pc == piece0) {  // the first chunk of the first piece comes with the CTA head
         pg_cur = head->first_pages[lane];
-        if (pg_cur >= d.n_pool_pages) {
+        if (c_cur * 32 + lane < rq.n_pages && (pg_cur < 0 || pg_cur >= d.n_pool_pages)) {
           d.status[0] = kDevBounds;
           d.status[1] = 201;
           pg_cur = 0;
@@ -589,7 +596,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant_
         const uint32_t stage = ring % kStages;
         ok = wait_bar(&ctrl->kv_empty[stage], ((ring / kStages) & 1u) ^ 1u, ctrl, d.status, 210);
         if (!ok) break;
-        if (lane == 0) mbar_arrive_expect_tx(&ctrl->kv_full[stage], (uint32_t)npages * 4096u);
+        if (lane == 0)
+          mbar_arrive_expect_tx(&ctrl->kv_full[stage], (uint32_t)npages * 4096u + ((blockIdx.x == 0 && ring == 0) ? tc.phantom_tx_bytes : 0u));
         __syncwarp();
         if (lane < 8 && page >= 0) {  // one 4 KB box per page: two 8-key groups x two d halves
           const uint32_t dst = smem_u32(kv_smem + stage * kTileBytes) + lane * 4096;
@@ -1286,6 +1294,8 @@ void tc_bind_device_plan(const TcHostPlan &h, unsigned char *image_base, unsigne
   t.n_cta = h.n_cta;
   t.n_targets = h.n_targets;
   t.tokens_per_mtile = h.tokens_per_mtile;
+  t.wait_limit_us = 1000000u;  // one second per wait
+  t.phantom_tx_bytes = 0;
   t.partial_ml = reinterpret_cast<float *>(scratch_base + h.s_ml);
   t.partial_o = reinterpret_cast<float *>(scratch_base + h.s_o);
 }

@@ -492,6 +492,26 @@ extern "C" int lr_plan_describe(const lr_plan *p, lr_plan_info *info) {
   return LR_OK;
 }
 
+extern "C" int lr_plan_debug_set_wait_limit(lr_plan *p, uint32_t microseconds) {
+  if (!p || microseconds == 0) {
+    set_error("lr_plan_debug_set_wait_limit: bad argument");
+    return LR_EINVAL;
+  }
+  p->tc.wait_limit_us = microseconds;
+  p->pr.wait_limit_us = microseconds;
+  return LR_OK;
+}
+
+extern "C" int lr_plan_debug_set_phantom_bytes(lr_plan *p, uint32_t bytes) {
+  if (!p) {
+    set_error("lr_plan_debug_set_phantom_bytes: null plan");
+    return LR_EINVAL;
+  }
+  p->tc.phantom_tx_bytes = bytes;
+  p->pr.phantom_tx_bytes = bytes;
+  return LR_OK;
+}
+
 extern "C" int lr_plan_debug_set_page(lr_plan *p, int32_t page_slot, int32_t new_id, void *stream) {
   if (!p || page_slot < 0 || page_slot >= p->dev.n_page_slots) {
     set_error("lr_plan_debug_set_page: bad argument");

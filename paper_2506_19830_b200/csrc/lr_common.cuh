@@ -104,6 +104,8 @@ struct DevTcPlan {
   const TcTarget *targets;
   int32_t n_cta, n_targets;
   int32_t tokens_per_mtile;  // floor(128 / group)
+  uint32_t wait_limit_us;    // bound of every device-side wait (test hook: lr_plan_debug_set_wait_limit)
+  uint32_t phantom_tx_bytes; // test hook: bytes CTA 0 expects on its first KV stage beyond what its copies deliver
   float *partial_o;          // [n_slots][32 chunks of 4 channels][128 rows][4] fp32, unnormalised
   float *partial_ml;         // [n_slots][128][2] (reference exponent in log2 units, sum)
 };
@@ -137,6 +139,7 @@ struct DevPairPlan {
   int32_t n_pairs, n_targets;
   int32_t tokens_per_mtile;
   uint32_t wait_limit_us;         // bound of every device-side wait (test hook: lr_plan_debug_set_wait_limit)
+  uint32_t phantom_tx_bytes;      // test hook: bytes CTA 0 of pair 0 expects on its first KV stage beyond what its copies deliver
   float *partial_o;               // [n_slots][32 chunks of 4 channels][128 rows][4] fp32, unnormalised
   float *partial_ml;              // [n_slots][128][2] (reference exponent in log2 units, sum)
   uint32_t *counters;             // [n_targets] arrival tickets of the contributors of a target; zero between launches

@@ -37,6 +37,8 @@ def _expect_bounds(plan, details):
     (2, B.PATH_TENSOR_CORE, (200, 201), lambda b: int(b.span_slot[0]) + 100),   # deep inside the prefix
     (2, B.PATH_TENSOR_CORE, (200, 201), lambda b: int(b.span_slot[0])),         # the first page a CTA fetches
     (2, B.PATH_TENSOR_CORE, (200, 201), lambda b: int(b.br_own_slot[1])),       # a branch tail
+    (2, B.PATH_PAIR, (200, 201), lambda b: int(b.span_slot[0]) + 100),
+    (2, B.PATH_PAIR, (200, 201), lambda b: int(b.span_slot[0])),
 ])
 def test_a_page_id_outside_the_pool_is_reported_not_dereferenced(cfg, path, details, slot_of):
     w = make_config(cfg, with_logits=False)
@@ -180,5 +182,35 @@ def test_compact_request_limit(n_req, ok):
         assert e.value.status == -2
         torch.cuda.synchronize()
         assert bool((new_len == -7).all()) and bool((n_kept == -7).all())  # refused before the first launch
+    plan.close()
+    ctx.close()
+
+
+@pytest.mark.parametrize("path", [B.PATH_TENSOR_CORE, B.PATH_PAIR])
+def test_a_wait_that_runs_out_is_reported_and_the_context_stays_usable(path):
+    """One barrier of the first CTA is made to expect bytes that never arrive, and the waits are given 3 ms instead of a
+    second: the CTA must give up, record LR_ETIMEOUT, drain what it has in flight and leave; the other CTAs finish;
+    the next pass on the same plan is correct."""
+    w = make_config(2, with_logits=False)
+    b, t = w.batch, w.tensors
+    ctx = B.Context(b.model, 0)
+    plan = B.Plan(ctx, b)
+    plan.lr_plan_set_attention_path(path)
+    x = R.DeviceInputs(b, t, DEV, with_logits=False)
+    buf, out, guard, n = _guarded_out(b)
+    plan.lr_plan_debug_set_wait_limit(3000)
+    plan.lr_plan_debug_set_phantom_bytes(4096)
+    plan.lr_verify_attention(x.q, x.k_pool, x.v_pool, out, None)
+    with pytest.raises(B.LrError) as e:
+        plan.lr_poll_status()
+    assert e.value.status == -4, e.value  # LR_ETIMEOUT
+    assert bool((buf[:guard] == -7.0).all()) and bool((buf[guard + n :] == -7.0).all())
+    plan.lr_plan_debug_set_phantom_bytes(0)
+    plan.lr_plan_debug_set_wait_limit(1_000_000)
+    for _ in range(2):
+        plan.lr_verify_attention(x.q, x.k_pool, x.v_pool, out, None)
+        assert plan.lr_poll_status() == 0
+    o_ref, _ = O.verify_attention(b, t.q, t.k_pool, t.v_pool)
+    check_attention(out, None, o_ref, None)
     plan.close()
     ctx.close()
