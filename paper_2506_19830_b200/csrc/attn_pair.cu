@@ -1041,23 +1041,21 @@ int pair_build_host_plan(const lr_ctx *ctx, const lr_batch *b, const int32_t *re
   const int n_q_rows = b->cu_q[b->n_branch];
   std::vector<TcPage> pages;
   std::vector<TcRow> rows((size_t)std::max(1, n_q_rows));
-  std::vector<TcReq> reqs((size_t)b->n_req);
+  std::vector<TcReq> reqs;  // one per page list (request x pair of M-tiles); PrPiece.req indexes it
   struct Grp { int req, kv, mtile0, n_mt, n_tiles, first_piece, n_pieces; };
   std::vector<Grp> grps;
+  // One page list per (request, pair of M-tiles): the prefix, the segments some branch of the group descends from and
+  // the tails of its own branches up to the last token one of its rows sees.  Pages no row of the group can see are
+  // left out, so no tile of the sweep is fully masked for everybody.
+  reqs.clear();
   for (int r = 0; r < b->n_req; ++r) {
     const int s0 = b->req_span_off[r], s1 = b->req_span_off[r + 1];
     const int br0 = req_br_off[r], br1 = req_br_off[r + 1];
-    TcReq &rq = reqs[r];
-    memset(&rq, 0, sizeof(rq));
-    rq.page_off = (int)pages.size();
     if (br1 == br0) continue;  // a request without branches has no query rows
     if (br1 - br0 > 254) return LR_OK;
-    rq.q_row0 = b->cu_q[br0];
-    rq.n_q = b->cu_q[br1] - b->cu_q[br0];
-    std::vector<unsigned char> node_used((size_t)(s1 - s0), 0);  // by depth-first number: some branch continues it
+    const int q_row0 = b->cu_q[br0], n_q = b->cu_q[br1] - b->cu_q[br0];
     for (int i = br0; i < br1; ++i) {
       const int tin = span_tin[s0 + b->br_depth[i]];
-      node_used[tin] = 1;
       if ((b->br_own_len[i] + kPage - 1) / kPage > 2047) return LR_OK;
       const int q_len = b->cu_q[i + 1] - b->cu_q[i];
       for (int k = 0; k < q_len; ++k) {
@@ -1066,30 +1064,48 @@ int pair_build_host_plan(const lr_ctx *ctx, const lr_batch *b, const int32_t *re
         w.limit = b->br_own_len[i] - q_len + k;
       }
     }
-    auto add_span = [&](int slot, int len, int need, int last, int owner) {
-      const int n = (len + kPage - 1) / kPage;
-      for (int p = 0; p < n; ++p) {
-        TcPage e;
-        e.page = b->page_ids[slot + p];
-        const uint32_t valid = (uint32_t)std::min(kPage, len - p * kPage);
-        e.meta = valid | ((uint32_t)need << 5) | ((uint32_t)owner << 13) | ((uint32_t)(owner ? p : last) << 21);
-        pages.push_back(e);
+    const int n_mtiles = (n_q + T - 1) / T;
+    for (int m0 = 0; m0 < n_mtiles; m0 += 2) {
+      const int mts = std::min(2, n_mtiles - m0);
+      const int row_lo = q_row0 + m0 * T, row_hi = q_row0 + std::min(n_q, (m0 + mts) * T);  // query rows of the group
+      TcReq rq;
+      memset(&rq, 0, sizeof(rq));
+      rq.page_off = (int)pages.size();
+      rq.q_row0 = q_row0;
+      rq.n_q = n_q;
+      std::vector<unsigned char> node_used((size_t)(s1 - s0), 0);  // by depth-first number: a branch of the group continues it
+      std::vector<int> tail_limit((size_t)(br1 - br0), -1);        // last tail token a row of the group sees, per branch
+      for (int i = br0; i < br1; ++i) {
+        const int lo = std::max(row_lo, b->cu_q[i]), hi = std::min(row_hi, b->cu_q[i + 1]);
+        if (lo >= hi) continue;
+        node_used[span_tin[s0 + b->br_depth[i]]] = 1;
+        tail_limit[i - br0] = rows[(size_t)hi - 1].limit;
       }
-    };
-    add_span(b->span_slot[s0], b->span_len[s0], 0, 255, 0);
-    rq.n_dense_tiles = (b->span_len[s0] / kPage) / kPagesPerTile;
-    for (int c = 1; s0 + c < s1; ++c) {  // a segment no branch sees is left out
-      bool seen = false;
-      for (int t = span_tin[s0 + c]; t <= span_last[s0 + c] && !seen; ++t) seen = node_used[t];
-      if (seen) add_span(b->span_slot[s0 + c], b->span_len[s0 + c], span_tin[s0 + c], span_last[s0 + c], 0);
+      auto add_span = [&](int slot, int len, int n_pg, int need, int last, int owner) {
+        for (int p = 0; p < n_pg; ++p) {
+          TcPage e;
+          e.page = b->page_ids[slot + p];
+          const uint32_t valid = (uint32_t)std::min(kPage, len - p * kPage);
+          e.meta = valid | ((uint32_t)need << 5) | ((uint32_t)owner << 13) | ((uint32_t)(owner ? p : last) << 21);
+          pages.push_back(e);
+        }
+      };
+      add_span(b->span_slot[s0], b->span_len[s0], (b->span_len[s0] + kPage - 1) / kPage, 0, 255, 0);
+      rq.n_dense_tiles = (b->span_len[s0] / kPage) / kPagesPerTile;
+      for (int c = 1; s0 + c < s1; ++c) {
+        bool seen = false;
+        for (int t = span_tin[s0 + c]; t <= span_last[s0 + c] && !seen; ++t) seen = node_used[t];
+        if (seen) add_span(b->span_slot[s0 + c], b->span_len[s0 + c], (b->span_len[s0 + c] + kPage - 1) / kPage, span_tin[s0 + c], span_last[s0 + c], 0);
+      }
+      for (int i = br0; i < br1; ++i)
+        if (tail_limit[i - br0] >= 0) add_span(b->br_own_slot[i], b->br_own_len[i], tail_limit[i - br0] / kPage + 1, 0, 0, i - br0 + 1);
+      rq.n_pages = (int)pages.size() - rq.page_off;
+      while (pages.size() % kPagesPerTile) pages.push_back(TcPage{0, 0});  // absent pages of the last tile: nothing valid
+      const int n_tiles = (rq.n_pages + kPagesPerTile - 1) / kPagesPerTile;
+      const int list = (int)reqs.size();
+      reqs.push_back(rq);
+      for (int kv = 0; kv < m.n_kv_heads; ++kv) grps.push_back(Grp{list, kv, m0, mts, n_tiles, 0, 0});
     }
-    for (int i = br0; i < br1; ++i) add_span(b->br_own_slot[i], b->br_own_len[i], 0, 0, i - br0 + 1);
-    rq.n_pages = (int)pages.size() - rq.page_off;
-    while (pages.size() % kPagesPerTile) pages.push_back(TcPage{0, 0});  // absent pages of the last tile: nothing valid
-    const int n_tiles = (rq.n_pages + kPagesPerTile - 1) / kPagesPerTile;
-    const int n_mtiles = (rq.n_q + T - 1) / T;
-    for (int kv = 0; kv < m.n_kv_heads; ++kv)
-      for (int m0 = 0; m0 < n_mtiles; m0 += 2) grps.push_back(Grp{r, kv, m0, std::min(2, n_mtiles - m0), n_tiles, 0, 0});
   }
   if (grps.empty()) return LR_OK;
   // Contiguous partition of the tile sequence (groups in order, tiles in order) over at most max_pairs pairs that
@@ -1205,6 +1221,7 @@ int pair_build_host_plan(const lr_ctx *ctx, const lr_batch *b, const int32_t *re
   out.o_pages = img.add(pages.data(), pages.size() * sizeof(TcPage));
   out.o_rows = img.add(rows.data(), rows.size() * sizeof(TcRow));
   out.o_pieces = img.add(pieces.data(), pieces.size() * sizeof(PrPiece));
+  if (reqs.empty()) reqs.push_back(TcReq{});
   out.o_reqs = img.add(reqs.data(), reqs.size() * sizeof(TcReq));
   if (targets.empty()) targets.push_back(TcTarget{});  // keep the section non-empty
   out.o_targets = img.add(targets.data(), targets.size() * sizeof(TcTarget));

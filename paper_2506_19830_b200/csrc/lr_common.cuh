@@ -69,14 +69,14 @@ struct TcRow {       // one per query row of the batch
   int32_t limit;         // last tail token the row sees
 };
 struct TcPiece {
-  int32_t req, kv_head;
+  int32_t req, kv_head;           // page list (index into reqs), KV head
   int32_t mtile0, n_mt;           // first M-tile and how many (1 or 2)
-  int32_t tile_begin, tile_end;   // tiles of the request's extended chain
+  int32_t tile_begin, tile_end;   // tiles of that page list
   int32_t slot[2];                // per stream: >= 0 partial slot, -1 write the final output, -2 nothing to write
 };
-struct TcReq {
-  int32_t page_off;     // first TcPage of the request
-  int32_t n_pages;      // extended-chain pages
+struct TcReq {           // one page list: what one group of M-tiles of a request sweeps (pieces index it by `req`)
+  int32_t page_off;     // first TcPage of the list
+  int32_t n_pages;      // its pages: prefix, the segments and tails some row of the group can see
   int32_t q_row0, n_q;  // query token range of the request
   int32_t n_dense_tiles;  // leading tiles made only of full prefix pages (no masking needed)
   int32_t pad[3];
