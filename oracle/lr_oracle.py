@@ -352,8 +352,33 @@ def sample_inverse_cdf(weights: np.ndarray, u: float) -> int:
     return int(np.searchsorted(c, u * c[-1], side="right"))
 
 
+def filter_probs(P: np.ndarray, top_k: int = 0, top_p: float = 1.0) -> np.ndarray:
+    """The sampling filters of Section 4, "Setup" (top_k 20, top_p 0.95 with the temperature): tokens are ranked by
+    probability, highest first, equal probabilities by lower index first.  top_k > 0 keeps the first top_k of the
+    ranking and renormalises; top_p < 1 then keeps the shortest leading part of the ranking whose mass reaches top_p
+    -- the token of rank r stays iff the tokens ranked before it hold less than top_p -- and renormalises again.
+    Returns the filtered distribution (zeros outside the kept set)."""
+    V = len(P)
+    order = np.lexsort((np.arange(V), -P))  # by probability descending, then index ascending
+    keep = np.ones(V, dtype=bool)
+    if top_k and top_k > 0:
+        keep[order[top_k:]] = False
+    P1 = np.where(keep, P, 0.0)
+    P1 = P1 / P1.sum()
+    if top_p < 1.0:
+        ranked = P1[order]
+        before = np.concatenate([[0.0], np.cumsum(ranked)[:-1]])  # mass of the tokens ranked ahead
+        stay = before < top_p
+        stay[0] = True
+        keep2 = np.zeros(V, dtype=bool)
+        keep2[order[stay]] = True
+        P1 = np.where(keep2, P1, 0.0)
+        P1 = P1 / P1.sum()
+    return P1
+
+
 def accept_sample(logits_bits: np.ndarray, draft_ids: np.ndarray, cu_draft: np.ndarray, temperature: float,
-                  u_accept: np.ndarray, u_final: np.ndarray):
+                  u_accept: np.ndarray, u_final: np.ndarray, top_k: int = 0, top_p: float = 1.0):
     """Rejection sampling of Background, "Speculative Decoding", for drafts whose draft distribution Q
     is a point mass at the drafted token (prompt-lookup / n-gram drafts, the paper's SD method):
 
@@ -362,8 +387,16 @@ def accept_sample(logits_bits: np.ndarray, draft_ids: np.ndarray, cu_draft: np.n
     token is sampled from the normalised max(0, P_i - Q_i), i.e. P_i with the rejected token removed;
     if every draft is accepted the final token is sampled from P of the extra row.  Sampling is by
     inverse CDF with u_final[b].  A draft id outside the vocabulary has probability 0.
+    With top_k > 0 or top_p < 1 the target distribution P_i is the filtered one (``filter_probs``): a draft
+    outside the kept set has probability 0 and is never accepted, and the final token comes from the kept set.
     Returns (n_accept, final_id, p_draft) with p_draft[i] = P_i(d_i).
     """
+    filtered = (top_k and top_k > 0) or top_p < 1.0
+
+    def probs(row):
+        P = target_probs(logits_bits[row], temperature)
+        return filter_probs(P, top_k, top_p) if filtered else P
+
     V = logits_bits.shape[1]
     B = len(cu_draft) - 1
     n_accept = np.zeros(B, dtype=np.int32)
@@ -375,7 +408,7 @@ def accept_sample(logits_bits: np.ndarray, draft_ids: np.ndarray, cu_draft: np.n
         n = 0
         residual = None
         while n < L:
-            P = target_probs(logits_bits[row0 + n], temperature)
+            P = probs(row0 + n)
             d = int(draft_ids[d0 + n])
             pd = P[d] if 0 <= d < V else 0.0
             p_draft[d0 + n] = pd
@@ -387,7 +420,7 @@ def accept_sample(logits_bits: np.ndarray, draft_ids: np.ndarray, cu_draft: np.n
                 residual[d] = 0.0
             break
         if residual is None:  # all accepted: one more token from the target
-            residual = target_probs(logits_bits[row0 + L], temperature)
+            residual = probs(row0 + L)
         n_accept[b] = n
         final_id[b] = sample_inverse_cdf(residual, float(u_final[b]))
     return n_accept, final_id, p_draft

@@ -957,12 +957,10 @@ attn_tc_merge_kernel(DevBatch d, DevTcPlan tc, uint16_t *__restrict__ out, float
   const int64_t qi = (int64_t)(g.q_row0 + tok) * d.n_q_heads + g.kv_head * G + r % G;
   const float2 *ml = reinterpret_cast<const float2 *>(tc.partial_ml) + (int64_t)g.slot_begin * 128 + r;
   const float4 *po = reinterpret_cast<const float4 *>(tc.partial_o) + ((int64_t)g.slot_begin * 32 + k) * 128 + r;
-  float M = -INFINITY;
-  for (int j = 0; j < g.n_slots; ++j) {
-    const float2 v = ml[(int64_t)j * 128];
-    if (v.y > 0.f) M = fmaxf(M, v.x);  // a stream that saw no key of the row contributes nothing
-  }
-  float L = 0.f;
+  // Eight slots at a time, the (exponent, sum) pairs and the partial outputs of a batch requested together: one
+  // round trip to memory per batch.  The running maximum moves between batches (never within one), in slot order,
+  // so the result depends on nothing but the partials.
+  float M = -INFINITY, L = 0.f;
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
   for (int j0 = 0; j0 < g.n_slots; j0 += 8) {
     float4 o[8];
@@ -970,9 +968,22 @@ attn_tc_merge_kernel(DevBatch d, DevTcPlan tc, uint16_t *__restrict__ out, float
 #pragma unroll
     for (int jj = 0; jj < 8; ++jj)
       if (j0 + jj < g.n_slots) {
-        o[jj] = po[(int64_t)(j0 + jj) * 32 * 128];
         v[jj] = ml[(int64_t)(j0 + jj) * 128];
+        o[jj] = po[(int64_t)(j0 + jj) * 32 * 128];
       }
+    float mb = M;
+#pragma unroll
+    for (int jj = 0; jj < 8; ++jj)
+      if (j0 + jj < g.n_slots && v[jj].y > 0.f) mb = fmaxf(mb, v[jj].x);  // a stream that saw no key of the row contributes nothing
+    if (mb > M) {
+      const float a = exp2f(M - mb);  // 0 while nothing has been accumulated (M = -inf)
+      L *= a;
+      acc.x *= a;
+      acc.y *= a;
+      acc.z *= a;
+      acc.w *= a;
+      M = mb;
+    }
 #pragma unroll
     for (int jj = 0; jj < 8; ++jj)
       if (j0 + jj < g.n_slots && v[jj].y > 0.f) {

@@ -116,3 +116,92 @@ def test_structural_invariants():
     n2, f2, _ = O.accept_sample(bits, drafts, cu, 0.7, ub, uf)
     assert np.array_equal(n, n2) and np.array_equal(f, f2)
     assert all(0 <= n[b] <= L for b in range(B)) and all(0 <= f[b] < V for b in range(B))
+
+
+# ---- the sampling filters (top_k, top_p) ---------------------------------------------------------------
+def test_filter_hand_computed_examples():
+    P = np.array([1 / 16, 1 / 2, 1 / 8, 1 / 4, 1 / 16])  # ranking: 1, 3, 2, then 0 before 4 (equal: lower index first)
+    # top_p = 0.8: ranks 0, 1, 2 have 0, 1/2, 3/4 ahead of them (< 0.8), rank 3 has 7/8: three tokens stay
+    assert O.filter_probs(P, 0, 0.8) == pytest.approx([0, 4 / 7, 1 / 7, 2 / 7, 0], abs=1e-15)
+    # exactly at a step: the tokens before rank 2 hold 3/4, which is not less than 3/4
+    assert O.filter_probs(P, 0, 0.75) == pytest.approx([0, 2 / 3, 0, 1 / 3, 0], abs=1e-15)
+    # top_k = 4 cuts between the two equal tokens: the lower index stays
+    assert O.filter_probs(P, 4, 1.0) == pytest.approx([1 / 15, 8 / 15, 2 / 15, 4 / 15, 0], abs=1e-15)
+    # both: after top_k = 2 the masses are 2/3, 1/3; top_p = 0.6 keeps only the first
+    assert O.filter_probs(P, 2, 0.6) == pytest.approx([0, 1, 0, 0, 0], abs=1e-15)
+    # no filter
+    assert np.array_equal(O.filter_probs(P, 0, 1.0), P)
+
+
+def test_filter_is_the_smallest_leading_set_that_reaches_top_p():
+    """Declarative check by brute force over sorted prefixes (independent of how the oracle walks the ranking)."""
+    rng = np.random.default_rng(5)
+    for trial in range(200):
+        V = int(rng.integers(2, 40))
+        P = rng.dirichlet(np.full(V, rng.choice([0.05, 0.3, 2.0])))
+        if trial % 3 == 0:  # ties
+            P = np.round(P * 16) + 1
+            P = P / P.sum()
+        k = int(rng.integers(0, V + 2))
+        p = float(rng.choice([0.3, 0.6, 0.9, 0.95, 0.999, 1.0]))
+        F = O.filter_probs(P, k, p)
+        kept = np.flatnonzero(F > 0)
+        ranked = sorted(range(V), key=lambda v: (-P[v], v))
+        n_k = min(k, V) if k > 0 else V
+        top = ranked[:n_k]
+        mass_k = sum(P[v] for v in top)
+        # smallest n with mass(first n) >= p * mass_k (all of them if none reaches it)
+        n_p = n_k
+        acc = 0.0
+        for n, v in enumerate(top, start=1):
+            acc += P[v]
+            if p < 1.0 and acc / mass_k >= p - 1e-15:
+                n_p = n
+                break
+        expect = sorted(top[:n_p])
+        if abs(sum(P[v] for v in top[:n_p - 1]) / mass_k - p) < 1e-12 or abs(acc / mass_k - p) < 1e-12:
+            continue  # a prefix mass within rounding of top_p: either side is a valid reading
+        assert list(kept) == expect, (trial, k, p)
+        assert F[kept] == pytest.approx(P[kept] / P[kept].sum(), rel=1e-12)  # renormalised, proportions unchanged
+
+
+def test_top_k_one_is_the_greedy_rule():
+    rng = np.random.default_rng(6)
+    V, L = 50, 5
+    rows = _bits(np.round(rng.standard_normal((L + 1, V)) * 2) / 2)  # coarse values: ties at the maximum happen
+    arg = O.row_argmax(rows)
+    cu = np.array([0, L], dtype=np.int32)
+    for trial in range(30):
+        drafts = arg[:L].astype(np.int32).copy()
+        miss = int(rng.integers(0, L + 1))
+        if miss < L:
+            drafts[miss] = (drafts[miss] + 1 + int(rng.integers(0, V - 1))) % V
+        ua, uf = rng.uniform(0, 0.999, L), rng.uniform(0, 1, 1)
+        n, f, p = O.accept_sample(rows, drafts, cu, 0.7, ua, uf, top_k=1)
+        n_ref, bonus_ref, _ = O.accept_greedy(rows, drafts, cu)
+        assert (n[0], f[0]) == (n_ref[0], bonus_ref[0])
+
+
+def test_filtered_output_distribution_equals_the_filtered_target():
+    """Exactness of speculative sampling with the filters on: the emitted token is distributed as the filtered P."""
+    rng = np.random.default_rng(7)
+    V, T = 7, 0.8
+    rows = _bits(rng.standard_normal((2, V)) * 1.5)
+    F = O.filter_probs(O.target_probs(rows[0], T), 5, 0.9)
+    assert 1 < (F > 0).sum() < V
+    cu = np.array([0, 1], dtype=np.int32)
+    n_grid = 2000
+    us = (np.arange(n_grid) + 0.5) / n_grid
+    kw = dict(top_k=5, top_p=0.9)
+    for d in range(V):
+        dd = np.array([d], dtype=np.int32)
+        # the acceptance decision depends on u_accept alone, the resampled token on u_final alone
+        acc = np.mean([O.accept_sample(rows, dd, cu, T, np.array([ua]), np.array([0.5]), **kw)[0][0] for ua in us])
+        hist = np.zeros(V)
+        for uf in us:
+            n, f, _ = O.accept_sample(rows, dd, cu, T, np.array([1.0]), np.array([uf]), **kw)
+            assert n[0] == 0
+            hist[f[0]] += 1
+        emitted = (1 - acc) * hist / n_grid
+        emitted[d] += acc
+        assert emitted == pytest.approx(F, abs=2e-3), d
