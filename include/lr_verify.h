@@ -254,6 +254,35 @@ int lr_accept_sample(lr_ctx *ctx, const void *logits_d, int64_t row_stride_elems
                      float *p_draft_d, void *scratch_d, void *stream);
 
 /*
+ * lr_accept_sample with the sampling filters of Section 4, "Setup" (top-p 0.95,
+ * and top-k 20 for one model family) applied to the target distribution first.
+ * Rank the tokens of a row by P_i, largest first, equal values by index.
+ *   top_k > 0: only the first top_k ranks stay, renormalised;
+ *   top_p < 1: of those, rank r stays iff the renormalised mass of the ranks
+ *              before it is below top_p (the first always stays); renormalised.
+ * P'_i is the result (0 outside the kept set), and the rule of
+ * lr_accept_sample runs on P'_i: draft i is accepted iff u_accept < P'_i(d_i),
+ * the final token comes from P'_{n_b} with the rejected token removed, or from
+ * P'_{L_b}.  top_k = 0 and top_p = 1 switch the respective filter off.
+ * Masses are rounded to multiples of 2^-40 of the row's largest one and summed
+ * as integers: results do not depend on summation order, and the final draw is
+ * exact given those masses.  A row whose kept set changes when top_p moves by
+ * a few parts in 10^6 may keep one token more or fewer than an exact
+ * evaluation.  p_draft_d (nullable, [sum L_b]) receives P'_i(d_i) of every
+ * draft; n_kept_d (nullable, [n_rows]) the size of every row's kept set.
+ * Rows, strides and alignment as for lr_accept_greedy; temperature > 0,
+ * top_k >= 0, 0 < top_p <= 1, else LR_EINVAL.  scratch_d:
+ * lr_accept_sample_filtered_scratch_bytes bytes, 8-byte aligned, no initial
+ * contents needed; calls sharing it must not overlap on the device.
+ */
+int lr_accept_sample_filtered_scratch_bytes(const lr_ctx *ctx, int32_t n_rows, size_t *bytes_out);
+int lr_accept_sample_filtered(lr_ctx *ctx, const void *logits_d, int64_t row_stride_elems, const int32_t *draft_ids_d,
+                              const int32_t *cu_draft_d, int32_t n_branch, int32_t n_rows, float temperature,
+                              int32_t top_k, float top_p, const float *u_accept_d, const float *u_final_d,
+                              int32_t *n_accept_d, int32_t *final_id_d, float *p_draft_d, int32_t *n_kept_d,
+                              void *scratch_d, void *stream);
+
+/*
  * lr_accept_greedy without a caller-provided scratch buffer.  (The paper has no
  * counterpart: this is a packaging variant of the call above, same results.)
  *

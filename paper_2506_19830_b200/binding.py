@@ -94,6 +94,8 @@ def lib() -> C.CDLL:
             "lr_accept_greedy_static": [vp, vp, i64, vp, vp, i32, i32, vp, vp, vp, vp],
             "lr_accept_sample_scratch_bytes": [vp, i32, C.POINTER(sz)],
             "lr_accept_sample": [vp, vp, i64, vp, vp, i32, i32, f32, vp, vp, vp, vp, vp, vp, vp],
+            "lr_accept_sample_filtered_scratch_bytes": [vp, i32, C.POINTER(sz)],
+            "lr_accept_sample_filtered": [vp, vp, i64, vp, vp, i32, i32, f32, i32, f32, vp, vp, vp, vp, vp, vp, vp, vp],
             "lr_commit": [vp] + [vp] * 10 + [vp],
             "lr_cycle_simulate_sync": [i32, i64, i64, vp, i64, C.POINTER(lr_cycle_stats)],
             "lr_cycle_simulate_async": [i32, i64, i64, vp, i64, C.POINTER(lr_cycle_stats)],
@@ -229,6 +231,24 @@ class Context:
         _check(lib().lr_accept_sample(self.handle, _ptr(logits), logits.stride(0), _ptr(draft_ids), _ptr(cu_draft), n_branch,
                                       logits.shape[0], float(temperature), _ptr(u_accept), _ptr(u_final), _ptr(n_accept),
                                       _ptr(final_id), _ptr(p_draft), _ptr(scratch), _stream_ptr(stream)), "lr_accept_sample")
+
+    def lr_accept_sample_filtered(self, logits: torch.Tensor, draft_ids: torch.Tensor, cu_draft: torch.Tensor,
+                                  temperature: float, top_k: int, top_p: float, u_accept: torch.Tensor, u_final: torch.Tensor,
+                                  n_accept: torch.Tensor, final_id: torch.Tensor, scratch: torch.Tensor,
+                                  p_draft: Optional[torch.Tensor] = None, n_kept: Optional[torch.Tensor] = None,
+                                  stream=None) -> None:
+        """``lr_accept_sample`` on the target distribution after the top-k / top-p filters (0 and 1.0 switch them off)."""
+        n_branch = cu_draft.numel() - 1
+        _check(lib().lr_accept_sample_filtered(self.handle, _ptr(logits), logits.stride(0), _ptr(draft_ids), _ptr(cu_draft),
+                                               n_branch, logits.shape[0], float(temperature), int(top_k), float(top_p),
+                                               _ptr(u_accept), _ptr(u_final), _ptr(n_accept), _ptr(final_id), _ptr(p_draft),
+                                               _ptr(n_kept), _ptr(scratch), _stream_ptr(stream)), "lr_accept_sample_filtered")
+
+    def accept_sample_filtered_scratch(self, n_rows: int) -> torch.Tensor:
+        n = C.c_size_t()
+        _check(lib().lr_accept_sample_filtered_scratch_bytes(self.handle, n_rows, C.byref(n)),
+               "lr_accept_sample_filtered_scratch_bytes")
+        return torch.empty((n.value + 7) // 8, dtype=torch.int64, device=f"cuda:{self.device}")
 
     def accept_sample_scratch(self, n_rows: int) -> torch.Tensor:
         n = C.c_size_t()

@@ -9,7 +9,7 @@ PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG_DIR, "csrc")
 INCLUDE = os.path.join(os.path.dirname(PKG_DIR), "include")
 LIB_PATH = os.path.join(PKG_DIR, "liblr_verify.so")
-SOURCES = ["lr_api.cu", "accept_greedy.cu", "accept_sample.cu", "commit.cu", "compact.cu", "cycle_host.cu", "attn_generic.cu", "attn_tc.cu", "attn_pair.cu"]
+SOURCES = ["lr_api.cu", "accept_greedy.cu", "accept_sample.cu", "accept_filter.cu", "commit.cu", "compact.cu", "cycle_host.cu", "attn_generic.cu", "attn_tc.cu", "attn_pair.cu"]
 
 
 def _nvcc() -> str:

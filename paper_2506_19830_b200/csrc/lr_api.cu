@@ -659,6 +659,42 @@ extern "C" int lr_accept_sample(lr_ctx *ctx, const void *logits, int64_t stride,
                               final_id, p_draft, scratch, reinterpret_cast<cudaStream_t>(stream));
 }
 
+extern "C" int lr_accept_sample_filtered_scratch_bytes(const lr_ctx *ctx, int32_t n_rows, size_t *bytes_out) {
+  if (!ctx || !bytes_out || n_rows < 0) {
+    set_error("lr_accept_sample_filtered_scratch_bytes: bad argument");
+    return LR_EINVAL;
+  }
+  *bytes_out = accept_filtered_scratch_bytes(n_rows);
+  return LR_OK;
+}
+
+extern "C" int lr_accept_sample_filtered(lr_ctx *ctx, const void *logits, int64_t stride, const int32_t *drafts,
+                                         const int32_t *cu_draft, int32_t n_branch, int32_t n_rows, float temperature,
+                                         int32_t top_k, float top_p, const float *u_accept, const float *u_final,
+                                         int32_t *n_accept, int32_t *final_id, float *p_draft, int32_t *n_kept, void *scratch,
+                                         void *stream) {
+  if (!ctx || !logits || !cu_draft || !u_final || !n_accept || !final_id || !scratch ||
+      ((!drafts || !u_accept) && n_rows > n_branch)) {
+    set_error("lr_accept_sample_filtered: null argument");
+    return LR_EINVAL;
+  }
+  if (n_branch < 0 || n_rows < n_branch) {
+    set_error("lr_accept_sample_filtered: n_rows %d < n_branch %d", n_rows, n_branch);
+    return LR_EINVAL;
+  }
+  if (!(temperature > 0.f) || top_k < 0 || !(top_p > 0.f) || top_p > 1.f) {
+    set_error("lr_accept_sample_filtered: temperature must be positive, top_k >= 0 (0 = off), top_p in (0, 1] (1 = off)");
+    return LR_EINVAL;
+  }
+  if (((uintptr_t)logits & 15) != 0 || (stride & 7) != 0 || stride < ctx->model.vocab || ((uintptr_t)scratch & 7) != 0) {
+    set_error("lr_accept_sample_filtered: logits must be 16-byte aligned with a row stride that is a multiple of 8 and >= vocab");
+    return LR_EINVAL;
+  }
+  if (n_branch == 0) return LR_OK;
+  return launch_accept_filtered(ctx, logits, stride, drafts, cu_draft, n_branch, n_rows, temperature, top_k, top_p, u_accept,
+                                u_final, n_accept, final_id, p_draft, n_kept, scratch, reinterpret_cast<cudaStream_t>(stream));
+}
+
 extern "C" int lr_commit(lr_plan *p, const uint8_t *verdict, const int32_t *n_accept, int32_t *n_steps, int32_t *survivor,
                          int32_t *committed, int32_t *keep_off, int32_t *keep_pages, int32_t *keep_valid,
                          int32_t *free_off, int32_t *free_pages, void *stream) {

@@ -270,6 +270,11 @@ size_t accept_sample_scratch_bytes(int32_t vocab, int32_t n_rows);
 int launch_accept_sample(lr_ctx *ctx, const void *logits, int64_t stride, const int32_t *drafts, const int32_t *cu_draft,
                          int32_t n_branch, int32_t n_rows, float temperature, const float *u_accept, const float *u_final,
                          int32_t *n_accept, int32_t *final_id, float *p_draft, void *scratch, cudaStream_t s);
+size_t accept_filtered_scratch_bytes(int32_t n_rows);
+int launch_accept_filtered(lr_ctx *ctx, const void *logits, int64_t stride, const int32_t *drafts, const int32_t *cu_draft,
+                           int32_t n_branch, int32_t n_rows, float temperature, int32_t top_k, float top_p,
+                           const float *u_accept, const float *u_final, int32_t *n_accept, int32_t *final_id, float *p_draft,
+                           int32_t *n_kept, void *scratch, cudaStream_t s);
 int launch_compact(lr_plan *p, const int32_t *keep_off, const int32_t *keep_pages, const int32_t *keep_valid, void *k_pool,
                    void *v_pool, int32_t *new_len, int32_t *n_pages_kept, void *scratch, cudaStream_t s);
 int launch_commit(lr_plan *p, const uint8_t *verdict, const int32_t *n_accept, int32_t *n_steps, int32_t *survivor,
