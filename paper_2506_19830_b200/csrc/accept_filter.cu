@@ -2,7 +2,8 @@
 // the target distribution before the rejection-sampling rule of Background, "Speculative Decoding".
 //
 // The filters keep a leading part of the ranking of a row's tokens by probability (descending; equal
-// probabilities in index order).  With bf16 logits the ranking is the ranking of a 16-bit ordered key, so the
+// probabilities in index order).  With bf16 logits the ranking is the ranking of a 16-bit ordered key (-0 and +0
+// sharing one), so the
 // kept set of a row is described by a cut: every token whose key is above cut_key, and of the tokens whose key
 // equals cut_key those with an index up to cut_idx.  filter_rows_kernel (one CTA per row) finds the cut:
 //   pass 0   row maximum m;
@@ -33,34 +34,40 @@ constexpr int kFT = 512;           // threads of filter_rows_kernel
 constexpr int kWin = 8192;         // keys per window
 constexpr int kPer = kWin / kFT;   // window positions per thread in the scan
 constexpr int kST = 1024;          // threads of accept_filtered_kernel
-constexpr float kFixScale = 1099511627776.f;  // 2^40
 typedef unsigned long long u64;
+constexpr int32_t kNoKey = INT32_MIN;
 
 struct RowCut {  // what the second kernel needs to know about a row (32 bytes)
-  float m;
-  uint32_t cut_key;
-  int32_t cut_idx;
+  float m;          // row maximum (finite: a row without a finite logit gets -3e38)
+  int32_t cut_key;  // key32 of the last kept group of equal logits; kNoKey: everything is kept
+  int32_t cut_idx;  // largest index kept inside that group
   int32_t n_kept;
-  u64 z_fix;
+  u64 z_fix;        // mass of the kept set
   u64 reserved;
 };
 
-// bf16 bit pattern, canonical: NaN counts as -inf, -0 as +0
-__device__ __forceinline__ uint32_t canon(uint32_t b) {
-  if ((b & 0x7FFFu) > 0x7F80u) return 0xFF80u;
-  return b == 0x8000u ? 0u : b;
+// Order-preserving key of a bf16 value given as fp32 bits (low 16 bits zero): sign-magnitude turned into two's
+// complement, so that a larger value has a larger key and -0 and +0 share key 0.  A multiple of 65536; key32 >> 16
+// ("key16") lies in [-32768, 32767].  A NaN lies beyond the infinities; its mass is 0 (below), so wherever it lands
+// it changes no sum.
+__device__ __forceinline__ int32_t key32(uint32_t f) {
+  const uint32_t s = (uint32_t)((int32_t)f >> 31);
+  return (int32_t)(((f & 0x7FFFFFFFu) ^ s) - s);
 }
-// order-preserving key of a bf16 value: larger value, larger key
-__device__ __forceinline__ uint32_t key_of(uint32_t b) { return (b & 0x8000u) ? (~b & 0xFFFFu) : (b | 0x8000u); }
-__device__ __forceinline__ uint32_t bits_of_key(uint32_t k) { return (k & 0x8000u) ? (k & 0x7FFFu) : (~k & 0xFFFFu); }
-// mass of a token in units of 2^-40 relative to the row maximum (at most 2^40)
-__device__ __forceinline__ u64 wfix_of(uint32_t b, float m, float k_log2) {
-  if (!(m > -INFINITY)) return 0;
-  const float x = __uint_as_float(b << 16);
-  return __float2ull_rn(exp2f((x - m) * k_log2) * kFixScale);
+__device__ __forceinline__ uint32_t f_of_key16(int32_t key16) {
+  return key16 >= 0 ? (uint32_t)key16 << 16 : (0x8000u | (uint32_t)(-key16)) << 16;
+}
+// mass of a token in units of 2^-40 relative to the row maximum (at most 2^40): a subtraction, a multiply-add, one
+// exponential, one conversion.  The conversion turns NaN into 0.
+__device__ __forceinline__ u64 wfix_of(uint32_t f, float m, float k_log2) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(fmaf(__uint_as_float(f) - m, k_log2, 40.f)));
+  u64 r;
+  asm("cvt.rni.u64.f32 %0, %1;" : "=l"(r) : "f"(y));
+  return r;
 }
 
-// f(e, b) for every token e of the row (b = canonical bf16 bits), threads striding over 16-byte vectors
+// f(e, bits) for every token e of the row (bits = the logit as fp32 bits), threads striding over 16-byte vectors
 template <int kT, class F>
 __device__ __forceinline__ void row_strided(const uint16_t *rp, int32_t vocab, F &&f) {
   const int32_t n_vec = vocab >> 3;
@@ -79,14 +86,14 @@ __device__ __forceinline__ void row_strided(const uint16_t *rp, int32_t vocab, F
         const uint32_t w[4] = {v[k].x, v[k].y, v[k].z, v[k].w};
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-          f(vi * 8 + 2 * j, canon(w[j] & 0xFFFFu));
-          f(vi * 8 + 2 * j + 1, canon(w[j] >> 16));
+          f(vi * 8 + 2 * j, w[j] << 16);
+          f(vi * 8 + 2 * j + 1, w[j] & 0xFFFF0000u);
         }
       }
     }
   }
   const int32_t e = n_vec * 8 + (int32_t)threadIdx.x;  // vocab not a multiple of 8
-  if (e < vocab) f(e, canon((uint32_t)__ldg(rp + e)));
+  if (e < vocab) f(e, (uint32_t)__ldg(rp + e) << 16);
 }
 
 // the same with every thread owning a contiguous range of the row, ranges in thread order: visiting threads in
@@ -108,14 +115,54 @@ __device__ __forceinline__ void row_blocked(const uint16_t *rp, int32_t vocab, F
         const uint32_t w[4] = {v[k].x, v[k].y, v[k].z, v[k].w};
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-          f(vi * 8 + 2 * j, canon(w[j] & 0xFFFFu));
-          f(vi * 8 + 2 * j + 1, canon(w[j] >> 16));
+          f(vi * 8 + 2 * j, w[j] << 16);
+          f(vi * 8 + 2 * j + 1, w[j] & 0xFFFF0000u);
         }
       }
     }
   }
   if (threadIdx.x == kT - 1)
-    for (int32_t e = n_vec * 8; e < vocab; ++e) f(e, canon((uint32_t)__ldg(rp + e)));
+    for (int32_t e = n_vec * 8; e < vocab; ++e) f(e, (uint32_t)__ldg(rp + e) << 16);
+}
+
+// maximum of a row, two bf16 at a time (max.bf16x2 returns the other operand when one is NaN); never below -3e38
+template <int kT>
+__device__ __forceinline__ float row_max(const uint16_t *rp, int32_t vocab, float *s_w) {
+  const int32_t n_vec = vocab >> 3;
+  const uint4 *vp = reinterpret_cast<const uint4 *>(rp);
+  constexpr uint32_t kNegInf2 = 0xFF80FF80u;
+  uint32_t a = kNegInf2, b = kNegInf2;
+  auto mx = [](uint32_t x, uint32_t y) {
+    uint32_t r;
+    asm("max.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(x), "r"(y));
+    return r;
+  };
+  for (int32_t v0 = 0; v0 < n_vec; v0 += 4 * kT) {
+    uint4 v[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const int32_t vi = v0 + k * kT + (int32_t)threadIdx.x;
+      v[k] = vi < n_vec ? __ldg(vp + vi) : make_uint4(kNegInf2, kNegInf2, kNegInf2, kNegInf2);
+    }
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      a = mx(a, mx(v[k].x, v[k].y));
+      b = mx(b, mx(v[k].z, v[k].w));
+    }
+  }
+  a = mx(a, b);
+  float m = fmaxf(__uint_as_float(a << 16), __uint_as_float(a & 0xFFFF0000u));
+  const int32_t e = n_vec * 8 + (int32_t)threadIdx.x;
+  if (e < vocab) m = fmaxf(m, __uint_as_float((uint32_t)__ldg(rp + e) << 16));
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
+  if ((threadIdx.x & 31) == 0) s_w[threadIdx.x >> 5] = m;
+  __syncthreads();
+  float r = s_w[0];
+#pragma unroll
+  for (int k = 1; k < kT / 32; ++k) r = fmaxf(r, s_w[k]);
+  __syncthreads();
+  return fmaxf(r, -3.0e38f);
 }
 
 // inclusive scan over the block in thread order; `total` receives the sum over the block
@@ -141,21 +188,8 @@ __device__ __forceinline__ T block_scan(T v, T *s_w, T &total) {
   return v + base;
 }
 
-template <int kT>
-__device__ __forceinline__ float block_max(float v, float *s_w) {
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xFFFFFFFFu, v, o));
-  if ((threadIdx.x & 31) == 0) s_w[threadIdx.x >> 5] = v;
-  __syncthreads();
-  float r = s_w[0];
-#pragma unroll
-  for (int k = 1; k < kT / 32; ++k) r = fmaxf(r, s_w[k]);
-  __syncthreads();
-  return r;
-}
-
 struct KeyCut {  // the last token kept: a key, and how many of the tokens with that key
-  uint32_t key;
+  int32_t key;         // key16
   uint32_t j;          // tokens of the key that are kept (>= 1 when found)
   uint32_t cnt_key;    // tokens of the key
   uint32_t cnt_above;  // tokens with a larger key
@@ -164,10 +198,10 @@ struct KeyCut {  // the last token kept: a key, and how many of the tokens with 
 };
 
 // A window of kWin consecutive keys, hi down to hi - kWin + 1: per-key token counts in shared memory (position d
-// is key hi - d), and what lies above the window.
+// is key hi - d; keys here are key16), and what lies above the window.
 struct Window {
   int32_t hi;
-  int32_t next_hi;     // the largest key below the window that occurs in the row; -1 if none
+  int32_t next_hi;     // the largest key below the window that occurs in the row; kNoKey if none
   uint32_t cnt_above;
   u64 mass_above;
   uint32_t cnt;        // tokens inside
@@ -204,23 +238,25 @@ __device__ __forceinline__ void build_window(FilterShared &sh, const uint16_t *r
                                              int32_t hi, Window &win, u64 &mass_below) {
   for (int i = threadIdx.x; i < kWin; i += kFT) sh.cnt[i] = 0;
   __syncthreads();
-  int32_t nh = -1;
+  int32_t nh = kNoKey;
   u64 rest = 0;
-  row_strided<kFT>(rp, vocab, [&](int32_t, uint32_t b) {
-    const int32_t key = (int32_t)key_of(b);
-    const int32_t d = hi - key;
-    if (d >= 0) {
-      if (d < kWin) {
+  const int32_t hi32 = hi * 65536;
+  row_strided<kFT>(rp, vocab, [&](int32_t, uint32_t f) {
+    const int32_t k32 = key32(f);
+    if (k32 <= hi32) {  // keys above the window were counted by an earlier pass (a NaN beyond +inf: never)
+      const uint32_t d = ((uint32_t)hi32 - (uint32_t)k32) >> 16;
+      if (d < (uint32_t)kWin) {
         atomicAdd(&sh.cnt[d], 1u);
       } else {
-        nh = max(nh, key);
-        if (kFirst) rest += wfix_of(b, m, k_log2);
+        nh = max(nh, k32);
+        if (kFirst) rest += wfix_of(f, m, k_log2);
       }
     }
   });
   __syncthreads();
   win.hi = hi;
-  win.next_hi = block_max_i32<kFT>(nh, sh.wi);
+  nh = block_max_i32<kFT>(nh, sh.wi);
+  win.next_hi = nh == kNoKey ? kNoKey : nh >> 16;
   if (kFirst) {
     u64 all;
     block_scan<kFT, u64>(rest, sh.w64, all);
@@ -237,8 +273,7 @@ struct Mine {
 };
 
 __device__ __forceinline__ u64 w_of_pos(const Window &win, int pos, float m, float k_log2) {
-  const int32_t key = win.hi - pos;
-  return key >= 0 ? wfix_of(bits_of_key((uint32_t)key), m, k_log2) : 0;
+  return wfix_of(f_of_key16(win.hi - pos), m, k_log2);
 }
 
 __device__ __forceinline__ void scan_window(FilterShared &sh, Window &win, Mine &me, float m, float k_log2) {
@@ -277,7 +312,7 @@ __device__ __forceinline__ KeyCut locate(FilterShared &sh, const Window &win, co
         const bool here = kByMass ? (w > 0 && mass + (u64)c * w >= t_rel) : (cnt + c >= k_rel);
         if (here) {
           KeyCut r;
-          r.key = (uint32_t)(win.hi - pos);
+          r.key = win.hi - pos;
           r.cnt_key = c;
           r.cnt_above = win.cnt_above + cnt;
           r.mass_above = win.mass_above + mass;
@@ -308,14 +343,12 @@ filter_rows_kernel(const uint16_t *__restrict__ logits, int64_t row_stride, int3
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
   // ---- pass 0: the row maximum
-  float mx = -INFINITY;
-  row_strided<kFT>(rp, vocab, [&](int32_t, uint32_t b) { mx = fmaxf(mx, __uint_as_float(b << 16)); });
   if (tid == 0) {
     sh.cut_idx = INT32_MAX;
     sh.cut.j = 0;
   }
-  const float m = block_max<kFT>(mx, sh.wf);
-  const int32_t key_top = (int32_t)key_of(canon(__float_as_uint(m) >> 16));
+  const float m = row_max<kFT>(rp, vocab, sh.wf);
+  const int32_t key_top = key32(__float_as_uint(m)) >> 16;
 
   // ---- pass 1: the window that starts at the largest key, and the mass of the whole row
   Window win;
@@ -323,13 +356,17 @@ filter_rows_kernel(const uint16_t *__restrict__ logits, int64_t row_stride, int3
   u64 mass_below = 0;
   win.cnt_above = 0;
   win.mass_above = 0;
-  build_window<true>(sh, rp, vocab, m, k_log2, key_top, win, mass_below);
+  const uint32_t cnt_total = (uint32_t)vocab;
+  const bool by_k = top_k > 0 && (uint32_t)top_k < cnt_total;
+  const bool by_p = top_p < 1.f;
+  // the mass of the whole row is needed only when top-k does not cut: else the mass of the top k takes its place
+  if (by_k) build_window<false>(sh, rp, vocab, m, k_log2, key_top, win, mass_below);
+  else build_window<true>(sh, rp, vocab, m, k_log2, key_top, win, mass_below);
   scan_window(sh, win, me, m, k_log2);
   const u64 mass_total = win.mass + mass_below;
-  const uint32_t cnt_total = (uint32_t)vocab;
 
   auto advance = [&]() -> bool {  // the next window down; false when nothing is left below
-    if (win.next_hi < 0) return false;
+    if (win.next_hi == kNoKey) return false;
     win.cnt_above += win.cnt;
     win.mass_above += win.mass;
     u64 unused;
@@ -338,11 +375,10 @@ filter_rows_kernel(const uint16_t *__restrict__ logits, int64_t row_stride, int3
     return true;
   };
 
-  const bool by_k = top_k > 0 && (uint32_t)top_k < cnt_total;
-  const bool by_p = top_p < 1.f;
   KeyCut cut;
   bool have_cut = false;
   u64 w_k = mass_total;  // mass of what top-k keeps
+  uint32_t n_all = cnt_total;
 
   if (by_k) {
     const uint32_t k = (uint32_t)top_k;
@@ -352,6 +388,9 @@ filter_rows_kernel(const uint16_t *__restrict__ logits, int64_t row_stride, int3
       cut = locate<false>(sh, win, me, k, 0, m, k_log2);
       have_cut = true;
       w_k = cut.mass_above + (u64)cut.j * cut.w_key;
+    } else {  // fewer than k tokens that are numbers: every window was visited, nothing is cut
+      w_k = win.mass_above + win.mass;
+      n_all = win.cnt_above + win.cnt;
     }
   }
   if (by_p && w_k > 0) {
@@ -380,13 +419,14 @@ filter_rows_kernel(const uint16_t *__restrict__ logits, int64_t row_stride, int3
   // ---- last pass, only when the cut splits a group of equal keys: the index of the last one kept
   if (have_cut && cut.j < cut.cnt_key) {
     uint32_t mine = 0;
-    row_blocked<kFT>(rp, vocab, [&](int32_t, uint32_t b) { mine += key_of(b) == cut.key ? 1u : 0u; });
+    const int32_t cut32 = cut.key * 65536;
+    row_blocked<kFT>(rp, vocab, [&](int32_t, uint32_t f) { mine += key32(f) == cut32 ? 1u : 0u; });
     uint32_t all;
     const uint32_t before = block_scan<kFT, uint32_t>(mine, sh.w32, all) - mine;
     if (before < cut.j && cut.j <= before + mine) {
       uint32_t seen = before;
-      row_blocked<kFT>(rp, vocab, [&](int32_t e, uint32_t b) {
-        if (key_of(b) == cut.key && ++seen == cut.j) sh.cut_idx = e;
+      row_blocked<kFT>(rp, vocab, [&](int32_t e, uint32_t f) {
+        if (key32(f) == cut32 && ++seen == cut.j) sh.cut_idx = e;
       });
     }
     __syncthreads();
@@ -394,17 +434,17 @@ filter_rows_kernel(const uint16_t *__restrict__ logits, int64_t row_stride, int3
   if (tid == 0) {
     RowCut rc;
     rc.m = m;
-    rc.cut_key = have_cut ? cut.key : 0u;
+    rc.cut_key = have_cut ? cut.key * 65536 : kNoKey;
     rc.cut_idx = sh.cut_idx;
-    rc.n_kept = have_cut ? (int32_t)(cut.cnt_above + cut.j) : (int32_t)cnt_total;
-    rc.z_fix = have_cut ? cut.mass_above + (u64)cut.j * cut.w_key : mass_total;
+    rc.n_kept = have_cut ? (int32_t)(cut.cnt_above + cut.j) : (int32_t)n_all;
+    rc.z_fix = have_cut ? cut.mass_above + (u64)cut.j * cut.w_key : w_k;
     rc.reserved = 0;
     cuts[row] = rc;
     if (n_kept_out != nullptr) n_kept_out[row] = rc.n_kept;
   }
 }
 
-__device__ __forceinline__ bool is_kept(uint32_t key, int32_t e, const RowCut &rc) {
+__device__ __forceinline__ bool is_kept(int32_t key, int32_t e, const RowCut &rc) {
   return key > rc.cut_key || (key == rc.cut_key && e <= rc.cut_idx);
 }
 
@@ -432,8 +472,8 @@ accept_filtered_kernel(const uint16_t *__restrict__ logits, int64_t row_stride, 
     const int32_t d = draft_ids[d0 + i];
     float p = 0.f;
     if (d >= 0 && d < vocab && rc.z_fix > 0) {
-      const uint32_t bts = canon((uint32_t)logits[(int64_t)(r0 + i) * row_stride + d]);
-      if (is_kept(key_of(bts), d, rc)) p = (float)wfix_of(bts, rc.m, k_log2) / (float)rc.z_fix;
+      const uint32_t f = (uint32_t)logits[(int64_t)(r0 + i) * row_stride + d] << 16;
+      if (is_kept(key32(f), d, rc)) p = (float)wfix_of(f, rc.m, k_log2) / (float)rc.z_fix;
     }
     if (p_draft != nullptr) p_draft[d0 + i] = p;
     if (!(u_accept[d0 + i] < p)) atomicMin(&s_n, i);
@@ -449,10 +489,10 @@ accept_filtered_kernel(const uint16_t *__restrict__ logits, int64_t row_stride, 
   if (n < L) {
     const int32_t d = draft_ids[d0 + n];
     if (d >= 0 && d < vocab) {
-      const uint32_t bts = canon((uint32_t)rp[d]);
-      if (is_kept(key_of(bts), d, rc)) {
+      const uint32_t f = (uint32_t)rp[d] << 16;
+      if (is_kept(key32(f), d, rc)) {
         dead = d;
-        w_dead = wfix_of(bts, rc.m, k_log2);
+        w_dead = wfix_of(f, rc.m, k_log2);
       }
     }
   }
@@ -462,7 +502,7 @@ accept_filtered_kernel(const uint16_t *__restrict__ logits, int64_t row_stride, 
   if (total > 0 && target >= total) target = total - 1;
   u64 mine = 0;
   row_blocked<kST>(rp, vocab, [&](int32_t e, uint32_t bts) {
-    if (e != dead && is_kept(key_of(bts), e, rc)) mine += wfix_of(bts, rc.m, k_log2);
+    if (e != dead && is_kept(key32(bts), e, rc)) mine += wfix_of(bts, rc.m, k_log2);
   });
   u64 all;
   const u64 before = block_scan<kST, u64>(mine, s_w64, all) - mine;
@@ -470,7 +510,7 @@ accept_filtered_kernel(const uint16_t *__restrict__ logits, int64_t row_stride, 
     u64 cum = before;
     bool done = false;
     row_blocked<kST>(rp, vocab, [&](int32_t e, uint32_t bts) {
-      if (!done && e != dead && is_kept(key_of(bts), e, rc)) {
+      if (!done && e != dead && is_kept(key32(bts), e, rc)) {
         cum += wfix_of(bts, rc.m, k_log2);
         if (cum > target) {
           s_final = e;

@@ -142,7 +142,7 @@ def test_ragged_small(seed):
     _check(t.logits, t.draft_ids, b.cu_draft, 0.8, top_k, top_p, ua, uf, got)
 
 
-@pytest.mark.parametrize("top_k,top_p", [(0, 0.3), (777, 1.0), (5000, 0.7), (0, 0.999)])
+@pytest.mark.parametrize("top_k,top_p", [(0, 0.3), (777, 1.0), (5000, 0.7), (0, 0.999), (20000, 1.0), (20000, 0.9)])
 def test_ties_special_values_and_long_chains(top_k, top_p):
     """Flat rows (the cut splits one large group of equal logits: the kept ones are the lowest indices), coarse rows
     (many groups of equal logits), -inf and NaN entries, out-of-range drafts, a vocabulary that is not a multiple of
