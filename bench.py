@@ -473,6 +473,14 @@ def extras(M):
     def sample_only(c):
         ctx.lr_accept_sample(M.lc[c], x0.draft_ids, x0.cu_draft, 0.6, u_acc, u_fin, samp_n, samp_f, samp_scratch, None, None)
 
+    filt_scratch = ctx.accept_sample_filtered_scratch(b.n_logit_rows)
+
+    def filtered_only(top_k, top_p):
+        def f(c):
+            ctx.lr_accept_sample_filtered(M.lc[c], x0.draft_ids, x0.cu_draft, 0.6, top_k, top_p, u_acc, u_fin, samp_n, samp_f,
+                                          filt_scratch, None, None, None)
+        return f
+
     # compaction moves tokens in place; every call with the same keep lists moves the same number of bytes
     cmp_k = [x0.k_pool.clone() for _ in range(2)]
     cmp_v = [x0.v_pool.clone() for _ in range(2)]
@@ -496,6 +504,13 @@ def extras(M):
     out["lr_accept_sample"] = {"us": us, "GB/s": acc_b / (us * 1e-6) / 1e9, "frac_of_hbm_peak": acc_b / (us * 1e-6) / 1e9 / hbm_peak,
                                "algorithmic_bytes": acc_b, "temperature": 0.6,
                                "note": "rejection-sampling acceptance; not part of the timed step"}
+    for top_k, top_p in ((20, 0.95), (0, 0.95)):  # the sampling settings of the paper's two model families
+        ms, _ = M.timed_median(M.make_runner(filtered_only(top_k, top_p)), min_total_ms=50.0)
+        us = 1e3 * ms / M.K
+        out[f"lr_accept_sample_filtered(top_k={top_k},top_p={top_p})"] = {
+            "us": us, "GB/s": acc_b / (us * 1e-6) / 1e9, "frac_of_hbm_peak": acc_b / (us * 1e-6) / 1e9 / hbm_peak,
+            "algorithmic_bytes": acc_b, "temperature": 0.6, "top_k": top_k, "top_p": top_p,
+            "note": "top-k / top-p filters, then rejection-sampling acceptance; not part of the timed step"}
     ms, _ = M.timed_median(M.make_runner(compact_only), min_total_ms=50.0)
     us = 1e3 * ms / M.K
     # tokens lr_compact displaces: those behind the first partly filled kept page of each request

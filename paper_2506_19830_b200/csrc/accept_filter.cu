@@ -30,7 +30,7 @@ namespace lr {
 
 namespace {
 
-constexpr int kFT = 512;           // threads of filter_rows_kernel
+constexpr int kFT = 1024;          // threads of filter_rows_kernel
 constexpr int kWin = 8192;         // keys per window
 constexpr int kPer = kWin / kFT;   // window positions per thread in the scan
 constexpr int kST = 1024;          // threads of accept_filtered_kernel
@@ -332,7 +332,7 @@ __device__ __forceinline__ KeyCut locate(FilterShared &sh, const Window &win, co
   return r;
 }
 
-__global__ void __launch_bounds__(kFT, 2)
+__global__ void __launch_bounds__(kFT, 1)
 filter_rows_kernel(const uint16_t *__restrict__ logits, int64_t row_stride, int32_t vocab, float k_log2, int32_t top_k,
                    float top_p, RowCut *__restrict__ cuts, int32_t *__restrict__ n_kept_out) {
   __shared__ FilterShared sh;
