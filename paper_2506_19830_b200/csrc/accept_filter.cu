@@ -127,7 +127,7 @@ __device__ __forceinline__ void row_blocked(const uint16_t *rp, int32_t vocab, F
 
 // maximum of a row, two bf16 at a time (max.bf16x2 returns the other operand when one is NaN); never below -3e38
 template <int kT>
-__device__ __forceinline__ float row_max(const uint16_t *rp, int32_t vocab, float *s_w) {
+__device__ __forceinline__ float row_max(const uint16_t *rp, int32_t vocab, float *s_w, float &thread_max) {
   const int32_t n_vec = vocab >> 3;
   const uint4 *vp = reinterpret_cast<const uint4 *>(rp);
   constexpr uint32_t kNegInf2 = 0xFF80FF80u;
@@ -154,6 +154,7 @@ __device__ __forceinline__ float row_max(const uint16_t *rp, int32_t vocab, floa
   float m = fmaxf(__uint_as_float(a << 16), __uint_as_float(a & 0xFFFF0000u));
   const int32_t e = n_vec * 8 + (int32_t)threadIdx.x;
   if (e < vocab) m = fmaxf(m, __uint_as_float((uint32_t)__ldg(rp + e) << 16));
+  thread_max = m;  // the largest logit among the tokens this thread looked at
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
   if ((threadIdx.x & 31) == 0) s_w[threadIdx.x >> 5] = m;
@@ -232,16 +233,18 @@ __device__ __forceinline__ int32_t block_max_i32(int32_t v, int32_t *s_w) {
 }
 
 // One pass over the row: counts of the keys inside the window starting at `hi`.  On the first window (kFirst) the
-// mass of everything below the window is summed too, so that the mass of the whole row is known.
+// mass of everything below the window is summed too, so that the mass of the whole row is known.  Tokens whose
+// logit is below `floor_x` are left out altogether (-inf: none is; a NaN always is).
 template <bool kFirst>
 __device__ __forceinline__ void build_window(FilterShared &sh, const uint16_t *rp, int32_t vocab, float m, float k_log2,
-                                             int32_t hi, Window &win, u64 &mass_below) {
+                                             float floor_x, int32_t hi, Window &win, u64 &mass_below) {
   for (int i = threadIdx.x; i < kWin; i += kFT) sh.cnt[i] = 0;
   __syncthreads();
   int32_t nh = kNoKey;
   u64 rest = 0;
   const int32_t hi32 = hi * 65536;
   row_strided<kFT>(rp, vocab, [&](int32_t, uint32_t f) {
+    if (!(__uint_as_float(f) >= floor_x)) return;
     const int32_t k32 = key32(f);
     if (k32 <= hi32) {  // keys above the window were counted by an earlier pass (a NaN beyond +inf: never)
       const uint32_t d = ((uint32_t)hi32 - (uint32_t)k32) >> 16;
@@ -347,7 +350,8 @@ filter_rows_kernel(const uint16_t *__restrict__ logits, int64_t row_stride, int3
     sh.cut_idx = INT32_MAX;
     sh.cut.j = 0;
   }
-  const float m = row_max<kFT>(rp, vocab, sh.wf);
+  float thread_max;
+  const float m = row_max<kFT>(rp, vocab, sh.wf, thread_max);
   const int32_t key_top = key32(__float_as_uint(m)) >> 16;
 
   // ---- pass 1: the window that starts at the largest key, and the mass of the whole row
@@ -359,9 +363,28 @@ filter_rows_kernel(const uint16_t *__restrict__ logits, int64_t row_stride, int3
   const uint32_t cnt_total = (uint32_t)vocab;
   const bool by_k = top_k > 0 && (uint32_t)top_k < cnt_total;
   const bool by_p = top_p < 1.f;
+  // With top-k on and k no larger than the number of threads, the k-th largest of the threads' own maxima (each is
+  // the logit of a different token) is a lower bound of the k-th largest logit of the row: tokens below it cannot be
+  // kept, and the passes that follow skip them after one comparison.
+  float floor_x = -INFINITY;
+  if (by_k && top_k <= kFT) {
+    for (int i = tid; i < kWin; i += kFT) sh.cnt[i] = 0;
+    __syncthreads();
+    const int32_t k32 = key32(__float_as_uint(thread_max));
+    const uint32_t d = ((uint32_t)(key_top * 65536) - (uint32_t)k32) >> 16;  // thread_max <= m
+    if (thread_max > -INFINITY && d < (uint32_t)kWin) atomicAdd(&sh.cnt[d], 1u);
+    __syncthreads();
+    win.hi = key_top;
+    scan_window(sh, win, me, m, k_log2);
+    if ((uint32_t)top_k <= win.cnt) {
+      const KeyCut kc = locate<false>(sh, win, me, (uint32_t)top_k, 0, m, k_log2);
+      floor_x = __uint_as_float(f_of_key16(kc.key));
+    }
+    __syncthreads();
+  }
   // the mass of the whole row is needed only when top-k does not cut: else the mass of the top k takes its place
-  if (by_k) build_window<false>(sh, rp, vocab, m, k_log2, key_top, win, mass_below);
-  else build_window<true>(sh, rp, vocab, m, k_log2, key_top, win, mass_below);
+  if (by_k) build_window<false>(sh, rp, vocab, m, k_log2, floor_x, key_top, win, mass_below);
+  else build_window<true>(sh, rp, vocab, m, k_log2, floor_x, key_top, win, mass_below);
   scan_window(sh, win, me, m, k_log2);
   const u64 mass_total = win.mass + mass_below;
 
@@ -370,7 +393,7 @@ filter_rows_kernel(const uint16_t *__restrict__ logits, int64_t row_stride, int3
     win.cnt_above += win.cnt;
     win.mass_above += win.mass;
     u64 unused;
-    build_window<false>(sh, rp, vocab, m, k_log2, win.next_hi, win, unused);
+    build_window<false>(sh, rp, vocab, m, k_log2, floor_x, win.next_hi, win, unused);
     scan_window(sh, win, me, m, k_log2);
     return true;
   };
@@ -404,7 +427,7 @@ filter_rows_kernel(const uint16_t *__restrict__ logits, int64_t row_stride, int3
       win.cnt_above = 0;
       win.mass_above = 0;
       u64 unused;
-      build_window<false>(sh, rp, vocab, m, k_log2, key_top, win, unused);
+      build_window<false>(sh, rp, vocab, m, k_log2, floor_x, key_top, win, unused);
       scan_window(sh, win, me, m, k_log2);
     }
     while (ok && t > win.mass_above + win.mass) ok = advance();
