@@ -3,6 +3,7 @@ the attention kernel in ``profiles/traffic.json``, which ``bench.py`` reads for 
 
     python -m paper_2506_19830_b200.ncu_summary report.ncu-rep --out profiles/attention_config3.txt \
         --title "lr_verify_attention on config 3" --command "ncu --set full ... python bench.py ..." \
+        [more reports, more --command lines] \
         [--traffic-workload config3_long_context --traffic-kernel attn_tc_kernel]
 
     python -m paper_2506_19830_b200.ncu_summary launches.csv --launch-list --out profiles/launch_list.txt ...
@@ -108,21 +109,22 @@ def record_traffic(launches, workload: str, kernel: str) -> None:
 
 def main() -> int:
     ap = argparse.ArgumentParser()
-    ap.add_argument("report")
+    ap.add_argument("report", nargs="+", help="one or more reports (their launches are listed one after another)")
     ap.add_argument("--out", required=True)
     ap.add_argument("--title", default="")
-    ap.add_argument("--command", default="", help="the full command that produced the report")
+    ap.add_argument("--command", action="append", default=[], help="the full command that produced a report (repeatable)")
     ap.add_argument("--note", action="append", default=[])
     ap.add_argument("--launch-list", action="store_true")
     ap.add_argument("--traffic-workload", default="")
     ap.add_argument("--traffic-kernel", default="attn_tc_kernel")
     a = ap.parse_args()
-    head = [f"# {a.title}", f"# command (B200, one GPU; preceded by the same command without ncu exiting 0):", f"#   {a.command}"]
+    head = [f"# {a.title}", "# command (B200, one GPU; each preceded by the same command without ncu exiting 0):"]
+    head += [f"#   {c}" for c in a.command]
     head += [f"# {n}" for n in a.note]
     if a.launch_list:
-        body = launch_list(a.report)
+        body = launch_list(a.report[0])
     else:
-        launches = read_report(a.report)
+        launches = [l for r in a.report for l in read_report(r)]
         body = summarise(launches)
         if a.traffic_workload:
             record_traffic(launches, a.traffic_workload, a.traffic_kernel)
