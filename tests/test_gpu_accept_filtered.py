@@ -206,3 +206,24 @@ def test_bad_arguments():
                                           z(1, torch.int32), z(1, torch.int32), scratch)
         assert e.value.status == -1  # LR_EINVAL
     ctx.close()
+
+
+@pytest.mark.parametrize("vocab,top_k,top_p", [(72, 8, 0.9), (72, 0, 0.5), (1000, 1024, 0.97), (3000, 1024, 1.0), (3000, 1025, 1.0),
+                                               (3000, 0, 1e-6), (40000, 2, 0.999)])
+def test_small_vocabularies_and_limits_of_the_bound(vocab, top_k, top_p):
+    """Vocabularies with fewer tokens than the filter kernel has threads (most threads see no token), top_k at and
+    just past the number of threads (the lower bound from the threads' maxima applies up to it), and a top_p so small
+    that only the most likely token stays."""
+    rng = np.random.default_rng(vocab + top_k)
+    L, nb = 6, 4
+    n_rows = nb * (L + 1)
+    bits = bf16_round((rng.standard_normal((n_rows, vocab)) * 3).astype(np.float32))
+    cu = np.arange(0, nb * L + 1, L, dtype=np.int32)
+    arg = O.row_argmax(bits)
+    drafts = np.where(rng.uniform(size=nb * L) < 0.6, np.concatenate([arg[b * (L + 1): b * (L + 1) + L] for b in range(nb)]),
+                      rng.integers(0, vocab, nb * L)).astype(np.int32)
+    ua, uf = rng.uniform(0, 1, nb * L), rng.uniform(0, 1, nb)
+    got = _run(Model(1, 1, 64, vocab), bits, drafts, cu, 0.7, top_k, top_p, ua, uf)
+    _check(bits, drafts, cu, 0.7, top_k, top_p, ua, uf, got, max_ambiguous_frac=0.5)
+    if top_p == 1e-6:
+        assert (got[3] == 1).all()
