@@ -1168,17 +1168,18 @@ int tc_build_host_plan(const lr_ctx *ctx, const lr_batch *b, const int32_t *req_
       const int n_tiles = (rq.n_pages + kPagesPerTile - 1) / kPagesPerTile;
       const int list = (int)reqs.size();
       reqs.push_back(rq);
-      for (int kv = 0; kv < m.n_kv_heads; ++kv) grps.push_back(Grp{list, kv, m0, mts, n_tiles, 1 + mts, 0, 0});
+      for (int kv = 0; kv < m.n_kv_heads; ++kv) grps.push_back(Grp{list, kv, m0, mts, n_tiles, mts == 2 ? 16 : 10, 0, 0});
     }
   }
   if (grps.empty()) return LR_OK;
   // Contiguous partition of the tile sequence (groups in order, tiles in order) over at most max_cta CTAs that
-  // minimises the largest CTA load.  A tile costs its group's weight; every piece -- a CTA's share of one group --
-  // costs kPieceStartTiles tiles more (Q load, pipeline ramp, epilogue), so a CTA that spans a group boundary gets
-  // fewer tiles; a tile that needs masks (anything past the full prefix pages) costs 8/5 of a dense one (measured).  For a load limit L the greedy fill (a CTA takes tiles while it stays within L) needs the fewest
+  // minimises the largest CTA load.  A tile costs its group's weight (10 with one M-tile, 16 with two: per-CTA cycle
+  // counts on the ragged serving workload gave 2360 and 3790 cycles a tile); every piece -- a CTA's share of one
+  // group -- costs kPieceStartTiles tiles more (Q load, pipeline ramp, epilogue: measured 1.7 to 1.8 tiles), so a CTA
+  // that spans a group boundary gets fewer tiles; a tile that needs masks (anything past the full prefix pages) costs 8/5 of a dense one (measured: 1.3 to 2.3 times, depending on the workload; 9/5 was no better).  For a load limit L the greedy fill (a CTA takes tiles while it stays within L) needs the fewest
   // CTAs possible; the smallest feasible L is found by bisection.  At most one CTA per two tiles: smaller shares
   // only add partial results to merge.
-  constexpr int kPieceStartTiles = 3, kDense = 5, kMasked = 8;  // costs in fifths of a dense tile
+  constexpr int kPieceStartTiles = 2, kDense = 5, kMasked = 8;  // costs in fifths of a dense tile
   auto tile_cost = [&](const Grp &g, int t) -> int64_t {
     return (int64_t)g.weight * (t >= reqs[g.req].n_dense_tiles ? kMasked : kDense);
   };
