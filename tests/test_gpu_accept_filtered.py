@@ -118,7 +118,7 @@ def _check(logits_bits, drafts, cu, T, top_k, top_p, ua, uf, got, max_ambiguous_
 
 # the paper's settings (Section 4, "Setup"): temperature 0.6 with top-p 0.95, and with top-k 20 besides
 @pytest.mark.parametrize("cfg,T,top_k,top_p", [(1, 0.6, 0, 0.95), (1, 0.6, 20, 0.95), (2, 0.6, 20, 0.95), (2, 0.6, 0, 0.95),
-                                               (2, 1.0, 50, 1.0)])
+                                               (2, 1.0, 50, 1.0), (3, 0.6, 0, 0.95), (5, 0.6, 20, 0.95)])
 def test_configs(cfg, T, top_k, top_p):
     w = make_config(cfg, with_kv=False)
     b, t = w.batch, w.tensors
